@@ -1,0 +1,211 @@
+/*
+ * rdk.h -- C ABI of the B200 (sm_100a) library for the hot path of the Redistributing Drafter
+ * Kernels (RDK) sampler of "Out-of-Vocabulary Sampling Boosts Speculative Decoding".
+ *
+ * For every row (one sequence at one draft position) the library
+ *   1. soft-maxes the pruned drafter's n logits and projects them onto the intersection with the
+ *      target vocabulary (Token-Level Intersection, Eq. "tli-drafter"; Algorithm 1 step 1) -> q',
+ *   2. redistributes q' onto the full target vocabulary of N tokens, either exactly,
+ *      w = M^T q' with a row-stochastic token-affinity matrix M (Algorithm 1 step 2, Eq.
+ *      "symbolic-m"), or with the linear-time first-order formula
+ *      theta = p^T q',  w_j = (N q'_j + theta p_j) / (N + p_j)   (Eq. "rdk-taylor"),
+ *      and normalises q~ = w / S, S = sum_j w_j,
+ *   3. draws a (possibly out-of-vocabulary) draft token d ~ q~, accepts it with probability
+ *      min(1, p_d / q~_d) and otherwise draws a replacement from the normalised residual
+ *      max(0, p - q~)   (Algorithm 1 step 3 = Algorithm 4 steps 4-8),
+ *   4. reports the closed-form acceptance rate alpha = sum_j min(p_j, q~_j) (Definition 2.1).
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The library allocates no
+ *     device memory and keeps no device state: inputs, outputs, the kept-id index, the affinity
+ *     matrix and workspaces are caller-owned and are neither freed nor retained after a call.
+ *   - Calls enqueue work on the caller's cudaStream_t (passed as void*; NULL = default stream) and
+ *     return at once; outputs are valid after the stream has been synchronised.  rdk_prepare_ids
+ *     and rdk_sample_and_verify_host are the exceptions: they synchronise the stream themselves.
+ *   - Every call returns an rdk_status.  Argument errors are detected on the host and launch
+ *     nothing.  There is no CPU fallback: on a device that is not compute capability 10.x every
+ *     compute call returns RDK_ERR_ARCH.
+ *   - A row index is r = b * positions + pos; per-(row, trial) outputs are indexed r * trials + t.
+ *   - Draws use the inverse CDF in ascending token id: the drawn token is the smallest j whose
+ *     inclusive prefix sum exceeds u * total, u in [0, 1).  Uniform lane 0 drives the draft draw,
+ *     lane 1 the acceptance test (accepted <=> u * q~_d < p_d), lane 2 the residual draw, lane 3
+ *     is spare.
+ */
+#ifndef RDK_H_
+#define RDK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum rdk_status {
+    RDK_OK = 0,
+    RDK_ERR_INVALID_ARG = 1,        /* null pointer, non-positive size, bad stride, bad enum      */
+    RDK_ERR_BAD_IDS = 2,            /* two drafter indices map to one target token                */
+    RDK_ERR_EMPTY_INTERSECTION = 3, /* no kept id lies in [0, N): the paper assumes I != {}       */
+    RDK_ERR_UNSUPPORTED = 4,        /* valid request that this build does not implement           */
+    RDK_ERR_WORKSPACE_TOO_SMALL = 5,
+    RDK_ERR_ARCH = 6,               /* current device is not sm_100                               */
+    RDK_ERR_CUDA = 7,               /* a CUDA call failed; text in rdk_last_error()               */
+    RDK_ERR_TIMEOUT = 8             /* a bounded device-side wait expired (read from status_word) */
+} rdk_status;
+
+typedef enum rdk_dtype { RDK_F32 = 0, RDK_BF16 = 1 } rdk_dtype;
+typedef enum rdk_kind { RDK_LOGITS = 0, RDK_PROBS = 1 } rdk_kind;
+typedef enum rdk_mode { RDK_MODE_LINEAR = 0, RDK_MODE_PRECOMPUTED_W = 1 } rdk_mode;
+
+/* Physical layouts of the affinity matrix M (n rows i in I, N columns j in T).
+ *   RDK_AFF_F32_ROWS : float  M[i * ld + j], ld >= N.           Contracted with fp32 FMAs.
+ *   RDK_AFF_BF16_COLS: bf16  Mt[j * ld + i], ld >= n, ld % 8 == 0, base 16-byte aligned
+ *                      (the transpose, so that the contraction index i is contiguous for both
+ *                      operands).  Contracted on the tensor cores with fp32 accumulation.      */
+typedef enum rdk_affinity_layout { RDK_AFF_F32_ROWS = 0, RDK_AFF_BF16_COLS = 1 } rdk_affinity_layout;
+
+typedef struct rdk_problem {
+    int32_t N;                  /* target vocabulary size |T|, >= 1                              */
+    int32_t n;                  /* drafter entries per row, >= 1                                 */
+    int32_t batch;              /* sequences                                                     */
+    int32_t positions;          /* draft positions per sequence; rows = batch * positions        */
+    int32_t target_dtype;       /* rdk_dtype of the target logits                                */
+    int32_t drafter_dtype;      /* rdk_dtype of the drafter logits / probabilities               */
+    int32_t drafter_kind;       /* rdk_kind: RDK_LOGITS are soft-maxed, RDK_PROBS taken as is    */
+    int32_t reserved;           /* must be 0                                                     */
+    int64_t target_row_stride;  /* elements between target rows; 0 means N                       */
+    int64_t drafter_row_stride; /* elements between drafter rows; 0 means n                      */
+    const void* kept_index;     /* device buffer filled by rdk_prepare_ids for this (N, n)       */
+} rdk_problem;
+
+typedef struct rdk_affinity {
+    const void* data;           /* device; layout as rdk_affinity_layout says                    */
+    int32_t layout;
+    int32_t reserved;           /* must be 0                                                     */
+    int64_t ld;                 /* leading dimension in elements                                 */
+} rdk_affinity;
+
+/* All members are device pointers, caller-allocated; any may be NULL (that output is skipped).  */
+typedef struct rdk_outputs {
+    int32_t* draft_token;       /* [rows * trials] d ~ q~ (may be outside the kept ids)          */
+    int32_t* out_token;         /* [rows * trials] d if accepted, else the residual draw         */
+    uint8_t* accepted;          /* [rows * trials] 1 / 0                                         */
+    float*   accept_prob;       /* [rows * trials] min(1, p_d / q~_d)                            */
+    float*   alpha;             /* [rows] sum_j min(p_j, q~_j)            (Definition 2.1)       */
+    float*   theta;             /* [rows] p^T q'  (linear mode only)                             */
+    float*   S;                 /* [rows] sum_j w_j                                              */
+    float*   residual_mass;     /* [rows] sum_j max(0, p_j - q~_j) = 1 - alpha  (Lemma 2.3)      */
+    int32_t* accepted_len;      /* [batch * trials] leading accepted positions (Alg. 4 step 7)   */
+    int32_t* status_word;       /* [1] device-side error code, 0 when fine; caller zeroes it     */
+} rdk_outputs;
+
+/* ---------------------------------------------------------------------------------------------
+ * Helpers
+ * ------------------------------------------------------------------------------------------- */
+int rdk_version(void);                          /* major * 1000 + minor                           */
+const char* rdk_status_string(int status);      /* static string, never NULL                      */
+const char* rdk_last_error(void);               /* thread-local detail of the last failure        */
+
+/* ---------------------------------------------------------------------------------------------
+ * Kept-id index.  The drafter's index i maps to target token kept_ids[i] (the intersection I of
+ * Sec. 2; ids < 0 or >= N stand for drafter tokens outside the target vocabulary, the set F, and
+ * are dropped by the TLI step).  rdk_prepare_ids validates the list and builds, in a caller-owned
+ * device buffer of rdk_kept_index_bytes(N, n) bytes (256-byte aligned), a membership bitmask over
+ * T with rank counts and the rank -> drafter-index table that the row kernels read.  Any order of
+ * ids is accepted; ascending valid ids are the fastest case.
+ *   kept_ids       device int32 [n]
+ *   n_valid_host   host int*, may be NULL: receives the number of ids inside [0, N)
+ * Synchronises `stream`.  Errors: RDK_ERR_BAD_IDS (duplicate id), RDK_ERR_EMPTY_INTERSECTION,
+ * RDK_ERR_WORKSPACE_TOO_SMALL, RDK_ERR_INVALID_ARG.
+ * ------------------------------------------------------------------------------------------- */
+size_t rdk_kept_index_bytes(int32_t N, int32_t n);
+int rdk_prepare_ids(const int32_t* kept_ids, int32_t n, int32_t N, void* kept_index,
+                    size_t kept_index_bytes, int* n_valid_host, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * rdk_build_affinity -- Eq. "symbolic-m" (Sec. 4, "Token-affinity priors"), with the covariance
+ * Omega replaced by the cosine similarity of token embeddings:
+ *   Omega_ij = <e_{kappa_i}, e_j> / (|e_{kappa_i}| |e_j|),
+ *   M_ij = exp(Omega_ij / tau) / sum_{k in T} exp(Omega_ik / tau),   i in I, j in T.
+ * One-time preprocessing (the paper: "calculated once at preprocessing time").
+ *   embeddings   device [N, d] of emb_dtype, row stride emb_row_stride elements (0 means d)
+ *   kept_ids     device int32 [n]; rows whose id is outside [0, N) are written as zeros
+ *   tau          > 0
+ *   M_out        device, layout / ld as in rdk_affinity (data member is ignored; M_out is used)
+ *   ws           device workspace of rdk_build_affinity_workspace_bytes(N, n, d) bytes
+ * Arithmetic: fp32 dot products and soft-max; the result is rounded to bf16 (nearest even) only
+ * when it is stored in the bf16 layout.
+ * ------------------------------------------------------------------------------------------- */
+size_t rdk_build_affinity_workspace_bytes(int32_t N, int32_t n, int32_t d);
+int rdk_build_affinity(const void* embeddings, int32_t emb_dtype, int32_t d, int64_t emb_row_stride,
+                       const int32_t* kept_ids, int32_t n, int32_t N, float tau,
+                       const rdk_affinity* M_desc, void* M_out, void* ws, size_t ws_bytes,
+                       void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * rdk_redistribute_exact -- Algorithm 1 steps 1-2:  q' = TLI(softmax(drafter)),  w = M^T q'.
+ *   drafter   device [rows, n] logits or probabilities (problem->drafter_kind / drafter_dtype)
+ *   M         affinity matrix; RDK_AFF_BF16_COLS runs on the tensor cores (q' is rounded to bf16
+ *             as the left operand, products accumulate in fp32), RDK_AFF_F32_ROWS uses fp32 FMAs
+ *   w_out     device float [rows, N] (row stride N): un-normalised weights
+ *   S_out     device float [rows] or NULL: S = sum_j w_j (q~ = w / S)
+ *   ws        device workspace of rdk_exact_workspace_bytes(problem, M->layout) bytes, 256-byte
+ *             aligned (holds the q' operand)
+ *   status_word device int32 [1] or NULL: set to RDK_ERR_TIMEOUT if a bounded wait inside the
+ *             tensor-core pipeline expires (the kernel then stops early and w_out is incomplete)
+ * ------------------------------------------------------------------------------------------- */
+size_t rdk_exact_workspace_bytes(const rdk_problem* problem, int32_t affinity_layout);
+int rdk_redistribute_exact(const rdk_problem* problem, const void* drafter, const rdk_affinity* M,
+                           float* w_out, float* S_out, void* ws, size_t ws_bytes,
+                           int32_t* status_word, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * rdk_redistribute_linear -- Eq. "rdk-taylor" written out to memory (the element-wise checkable
+ * form of the linear path; rdk_sample_and_verify never stores this N-long vector).
+ *   target      device [rows, N] target logits (p = softmax(target))
+ *   drafter     device [rows, n]
+ *   qtilde_out  device float [rows, N] (row stride N): q~ = w / S
+ *   theta_out   device float [rows] or NULL
+ *   S_out       device float [rows] or NULL
+ * ------------------------------------------------------------------------------------------- */
+int rdk_redistribute_linear(const rdk_problem* problem, const void* target, const void* drafter,
+                            float* qtilde_out, float* theta_out, float* S_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * rdk_sample_and_verify -- Algorithm 1 step 3 / Algorithm 4 steps 4-8 for every row, fused with
+ * the redistribution that feeds it.
+ *   mode RDK_MODE_LINEAR:        q~ from Eq. "rdk-taylor", computed on the fly from target and
+ *                                drafter (w is never stored); `w` must be NULL.
+ *   mode RDK_MODE_PRECOMPUTED_W: q~ = w / sum(w) with w float [rows, N], row stride w_row_stride
+ *                                elements (0 means N), e.g. from rdk_redistribute_exact;
+ *                                `drafter` is ignored.
+ *   target     device [rows, N] target logits
+ *   uniforms   device float [rows, trials, 4] in [0, 1)
+ *   trials     >= 1 independent draws per row (each uses its own 4 uniforms)
+ *   out        see rdk_outputs
+ * ------------------------------------------------------------------------------------------- */
+int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* target,
+                          const void* drafter, const float* w, int64_t w_row_stride,
+                          const float* uniforms, int32_t trials, const rdk_outputs* out,
+                          void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * rdk_sample_and_verify_host -- the same step (linear mode) for callers whose logits live in HOST
+ * memory: copies target_host / drafter_host / uniforms_host to the caller's device staging
+ * buffers, runs rdk_sample_and_verify, copies the per-(row, trial) and per-row results back and
+ * synchronises the stream.  Host buffers should be pinned for full copy speed.
+ *   problem->kept_index, staging buffers: device.   *_host: host.
+ *   stage_target [rows * N], stage_drafter [rows * n] of the problem's dtypes, stage_uniforms
+ *   float [rows * trials * 4], dev_out: device outputs as in rdk_outputs (members that are NULL
+ *   are skipped, also in host_out); host_out: host arrays of the same shapes.
+ * ------------------------------------------------------------------------------------------- */
+int rdk_sample_and_verify_host(const rdk_problem* problem, const void* target_host,
+                               const void* drafter_host, const float* uniforms_host,
+                               int32_t trials, void* stage_target, void* stage_drafter,
+                               float* stage_uniforms, const rdk_outputs* dev_out,
+                               const rdk_outputs* host_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RDK_H_ */

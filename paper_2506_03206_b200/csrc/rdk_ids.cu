@@ -1,0 +1,141 @@
+// Kept-id index: membership bitmask over the target vocabulary, per-word rank counts and the
+// rank -> drafter-index table.  The intersection I = T n D of Sec. 2 is "ids inside [0, N)";
+// everything else is the out-of-vocabulary set F that Token-Level Intersection drops.
+#include "rdk_common.cuh"
+
+namespace rdk {
+
+__global__ void idx_clear_kernel(int32_t* header, uint32_t* mask, int32_t* slot, int words, int N, int n) {
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    const int stride = gridDim.x * blockDim.x;
+    for (int w = g; w < words; w += stride) mask[w] = 0u;
+    for (int i = g; i < n; i += stride) slot[i] = -1;
+    if (g == 0) {
+        for (int k = 0; k < 64; ++k) header[k] = 0;
+        header[kHdrN] = N;
+        header[kHdrn] = n;
+        header[kHdrIdentity] = 1;
+    }
+}
+
+__global__ void idx_mark_kernel(const int32_t* __restrict__ ids, int32_t* ids_copy, int32_t* header,
+                                uint32_t* mask, int N, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int id = ids[i];
+    ids_copy[i] = id;
+    if (id >= 0 && id < N) {
+        const uint32_t bit = 1u << (id & 31);
+        const uint32_t old = atomicOr(&mask[id >> 5], bit);
+        if (old & bit) atomicExch(&header[kHdrDup], 1);
+        atomicAdd(&header[kHdrValid], 1);
+    }
+}
+
+// One CTA: exclusive prefix sum of the per-word popcounts.
+__global__ void idx_rank_kernel(const uint32_t* __restrict__ mask, int32_t* rank, int words) {
+    __shared__ int warp_tot[32];
+    __shared__ int carry;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int w0 = 0; w0 < words; w0 += blockDim.x) {
+        const int w = w0 + threadIdx.x;
+        const int c = (w < words) ? __popc(mask[w]) : 0;
+        int incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) warp_tot[wid] = incl;
+        __syncthreads();
+        int before = carry;
+        for (int k = 0; k < wid; ++k) before += warp_tot[k];
+        if (w < words) rank[w] = before + incl - c;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int t = carry;
+            for (int k = 0; k < nw; ++k) t += warp_tot[k];
+            carry = t;
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void idx_slot_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ mask,
+                                const int32_t* __restrict__ rank, int32_t* slot, int32_t* header,
+                                int N, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int id = ids[i];
+    if (id < 0 || id >= N) {
+        atomicExch(&header[kHdrIdentity], 0);   // a dropped entry shifts every later rank
+        return;
+    }
+    const uint32_t word = mask[id >> 5];
+    const int r = rank[id >> 5] + __popc(word & ((1u << (id & 31)) - 1u));
+    slot[r] = i;                                 // duplicates (rejected by the host) would collide here
+    if (r != i) atomicExch(&header[kHdrIdentity], 0);
+}
+
+__global__ void idx_seal_kernel(int32_t* header) { header[kHdrMagic] = kIdxMagic; }
+
+}  // namespace rdk
+
+using namespace rdk;
+
+extern "C" size_t rdk_kept_index_bytes(int32_t N, int32_t n) {
+    if (N < 1 || n < 1) return 0;
+    return idx_bytes(N, n);
+}
+
+extern "C" int rdk_prepare_ids(const int32_t* kept_ids, int32_t n, int32_t N, void* kept_index,
+                               size_t kept_index_bytes, int* n_valid_host, void* stream) {
+    if (!kept_ids || !kept_index || N < 1 || n < 1) {
+        set_error("rdk_prepare_ids: null pointer or non-positive size (N=%d n=%d)", N, n);
+        return RDK_ERR_INVALID_ARG;
+    }
+    if ((reinterpret_cast<uintptr_t>(kept_index) & 255u) != 0) {
+        set_error("rdk_prepare_ids: kept_index must be 256-byte aligned");
+        return RDK_ERR_INVALID_ARG;
+    }
+    if (kept_index_bytes < idx_bytes(N, n)) {
+        set_error("rdk_prepare_ids: buffer has %zu bytes, %zu needed", kept_index_bytes, idx_bytes(N, n));
+        return RDK_ERR_WORKSPACE_TOO_SMALL;
+    }
+    const int st = check_arch();
+    if (st != RDK_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    KeptIndexView v = make_view(kept_index, N, n);
+    int32_t* header = const_cast<int32_t*>(v.header);
+    uint32_t* mask = const_cast<uint32_t*>(v.mask);
+    int32_t* rank = const_cast<int32_t*>(v.rank);
+    int32_t* slot = const_cast<int32_t*>(v.slot);
+    int32_t* ids = const_cast<int32_t*>(v.ids);
+    const int tb = 256;
+    const int work = v.words > n ? v.words : n;
+    int blocks = (work + tb - 1) / tb;
+    if (blocks > 1184) blocks = 1184;
+    idx_clear_kernel<<<blocks, tb, 0, s>>>(header, mask, slot, v.words, N, n);
+    idx_mark_kernel<<<(n + tb - 1) / tb, tb, 0, s>>>(kept_ids, ids, header, mask, N, n);
+    idx_rank_kernel<<<1, 1024, 0, s>>>(mask, rank, v.words);
+    idx_slot_kernel<<<(n + tb - 1) / tb, tb, 0, s>>>(ids, mask, rank, slot, header, N, n);
+    RDK_CUDA(cudaGetLastError());
+    int32_t host_hdr[8] = {0};
+    RDK_CUDA(cudaMemcpyAsync(host_hdr, header, sizeof(host_hdr), cudaMemcpyDeviceToHost, s));
+    RDK_CUDA(cudaStreamSynchronize(s));
+    if (n_valid_host) *n_valid_host = host_hdr[kHdrValid];
+    if (host_hdr[kHdrDup]) {
+        set_error("rdk_prepare_ids: two drafter indices map to the same target token");
+        return RDK_ERR_BAD_IDS;
+    }
+    if (host_hdr[kHdrValid] == 0) {
+        set_error("rdk_prepare_ids: no kept id lies inside the target vocabulary [0, %d)", N);
+        return RDK_ERR_EMPTY_INTERSECTION;
+    }
+    idx_seal_kernel<<<1, 1, 0, s>>>(header);
+    RDK_CUDA(cudaGetLastError());
+    RDK_CUDA(cudaStreamSynchronize(s));
+    return RDK_OK;
+}

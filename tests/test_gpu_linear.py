@@ -1,0 +1,181 @@
+"""GPU parity of the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8) against the CPU
+checker, through the C ABI, on the same seeded inputs and the same Philox uniforms."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import rdk_oracle as O
+import parity_util as PU
+
+pytestmark = pytest.mark.gpu
+
+KIND = {"logits": 0, "probs": 1}
+
+
+def _rdk():
+    import paper_2506_03206_b200 as rdk
+    return rdk
+
+
+def _run_linear(cfg, inp, rows=None, check_qtilde=True, kept_override=None):
+    rdk = _rdk()
+    B = rdk.binding
+    dev = "cuda"
+    kid = (kept_override if kept_override is not None else inp["kept_ids"]).to(dev)
+    idx = rdk.rdk_prepare_ids(kid, cfg.N)
+    target, drafter, uni = inp["target"].to(dev), inp["drafter"].to(dev), inp["uniforms"].to(dev)
+    kind = KIND[cfg.drafter_kind]
+    out = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, target, drafter, None, uni, cfg.batch,
+                                    cfg.positions, kind)
+    torch.cuda.synchronize()
+    B.check_status_word(out)
+    rows = list(range(cfg.rows)) if rows is None else rows
+    kappa = kid.cpu().numpy()
+    tally = PU.compare_sampling(inp, out, rows, "linear", kept_ids=kappa)
+    PU.compare_accepted_len(out, cfg.batch, cfg.positions, cfg.trials)
+    if check_qtilde:
+        qt, theta, S = rdk.rdk_redistribute_linear(idx, target, drafter, cfg.batch, cfg.positions, kind)
+        torch.cuda.synchronize()
+        refs = {}
+        for r in rows:
+            refs[r] = O.rdk_row(W.to_f64(inp["target"][r]), W.to_f64(inp["drafter"][r]), kappa,
+                                np.zeros((1, 4)), "linear", drafter_kind=cfg.drafter_kind)
+            assert PU.close(float(theta[r]), refs[r]["theta"], cfg.dtype == "bf16")
+            assert PU.close(float(S[r]), refs[r]["S"], cfg.dtype == "bf16")
+        PU.compare_qtilde(qt, refs, cfg.dtype == "bf16")
+    print(cfg.name, tally.summary())
+    return tally
+
+
+def test_config1_tiny_rdk_linear():
+    cfg = W.CONFIGS["C1"]
+    _run_linear(cfg, W.make_inputs(cfg)).assert_ok()
+
+
+@pytest.mark.parametrize("N,n", [(2, 1), (2, 2), (16, 1), (16, 4), (16, 16), (17, 5), (1000, 77),
+                                 (4096, 512), (4097, 1), (12289, 3000)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_shapes_linear(N, n, dtype):
+    cfg = W.tiny_config(N=N, n=n, rows=5, dtype=dtype, trials=16, seed=N * 31 + n)
+    _run_linear(cfg, W.make_inputs(cfg)).assert_ok(max_ambiguous_frac=0.1)
+
+
+def test_probability_drafter_linear():
+    cfg = W.tiny_config(N=3000, n=700, rows=4, dtype="bf16", trials=8, drafter_kind="probs", rho=0.8)
+    _run_linear(cfg, W.make_inputs(cfg)).assert_ok()
+    cfg = W.tiny_config(N=515, n=100, rows=3, dtype="f32", trials=8, drafter_kind="probs", rho=0.8)
+    _run_linear(cfg, W.make_inputs(cfg)).assert_ok()
+
+
+def test_zipf_pruned_mid_size_spans_several_tiles():
+    # several 4096-token tiles plus a ragged tail, Zipf-ranked kept ids, correlated logits
+    cfg = W.tiny_config(N=3 * 4096 + 1032, n=3300, rows=6, dtype="bf16", trials=4, kept_rule="zipf",
+                        zipf_bias=True, rho=0.8, seed=11)
+    _run_linear(cfg, W.make_inputs(cfg)).assert_ok()
+
+
+def test_unsorted_and_out_of_vocabulary_ids():
+    cfg = W.tiny_config(N=2000, n=300, rows=4, dtype="f32", trials=8, seed=5)
+    inp = W.make_inputs(cfg)
+    g = torch.Generator().manual_seed(3)
+    ids = inp["kept_ids"][torch.randperm(cfg.n, generator=g)].clone()    # any order is accepted
+    ids[7] = -1                                                          # drafter tokens outside T
+    ids[100] = cfg.N + 5
+    ids[299] = cfg.N
+    t = _run_linear(cfg, inp, kept_override=ids)
+    t.assert_ok()
+
+
+def test_strided_rows_and_unaligned_rows():
+    rdk = _rdk()
+    B = rdk.binding
+    cfg = W.tiny_config(N=1001, n=99, rows=4, dtype="bf16", trials=4, seed=9)   # odd N: rows not 16-byte aligned
+    _run_linear(cfg, W.make_inputs(cfg)).assert_ok()
+    # rows embedded in a wider buffer (row stride > N)
+    inp = W.make_inputs(cfg)
+    wide = torch.zeros(cfg.rows, cfg.N + 23, dtype=torch.bfloat16)
+    wide[:, : cfg.N] = inp["target"]
+    idx = rdk.rdk_prepare_ids(inp["kept_ids"].cuda(), cfg.N)
+    tgt = wide.cuda()[:, : cfg.N]
+    out = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, tgt, inp["drafter"].cuda(), None,
+                                    inp["uniforms"].cuda(), cfg.batch, cfg.positions)
+    torch.cuda.synchronize()
+    PU.compare_sampling(inp, out, range(cfg.rows), "linear").assert_ok()
+
+
+def test_directed_out_of_vocabulary_draw():
+    # Aim the draft uniform into the CDF interval of a pruned token: the sampler must return it.
+    rdk = _rdk()
+    B = rdk.binding
+    for N, n in [(16, 4), (64, 8)]:
+        cfg = W.tiny_config(N=N, n=n, rows=6, dtype="f32", trials=4, seed=N)
+        inp = W.make_inputs(cfg)
+        kappa = inp["kept_ids"].numpy()
+        oov = np.setdiff1d(np.arange(N), kappa)
+        u = inp["uniforms"].clone()
+        wanted = []
+        for r in range(cfg.rows):
+            ref = O.rdk_row(W.to_f64(inp["target"][r]), W.to_f64(inp["drafter"][r]), kappa, np.zeros((1, 4)), "linear")
+            j = int(oov[np.argmax(ref["w"][oov])])
+            lo = ref["cdf_w"][j - 1] if j else 0.0
+            mid = 0.5 * (lo + ref["cdf_w"][j]) / ref["S"]
+            u[r, :, 0] = float(np.float32(mid))
+            wanted.append(j)
+        inp["uniforms"] = u
+        idx = rdk.rdk_prepare_ids(inp["kept_ids"].cuda(), N)
+        out = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, inp["target"].cuda(), inp["drafter"].cuda(),
+                                        None, u.cuda(), cfg.batch, cfg.positions)
+        torch.cuda.synchronize()
+        t = PU.compare_sampling(inp, out, range(cfg.rows), "linear")
+        t.assert_ok()
+        d = out["draft_token"].cpu().numpy().reshape(cfg.rows, cfg.trials)
+        hits = sum(int(d[r, 0] == wanted[r]) for r in range(cfg.rows))
+        assert hits >= cfg.rows - 1 and all(w not in kappa for w in wanted)
+
+
+def test_identical_distributions_fall_back_to_p_for_the_residual():
+    # N = 1: q~ = p = [1]; the residual mass is 0, every draft is accepted with probability 1
+    rdk = _rdk()
+    B = rdk.binding
+    cfg = W.tiny_config(N=1, n=1, rows=2, dtype="f32", trials=4)
+    inp = W.make_inputs(cfg)
+    inp["kept_ids"] = torch.zeros(1, dtype=torch.int32)
+    idx = rdk.rdk_prepare_ids(inp["kept_ids"].cuda(), 1)
+    out = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, inp["target"].cuda(), inp["drafter"].cuda(), None,
+                                    inp["uniforms"].cuda(), cfg.batch, cfg.positions)
+    torch.cuda.synchronize()
+    assert torch.all(out["draft_token"] == 0) and torch.all(out["out_token"] == 0)
+    assert torch.all(out["accepted"] == 1)
+    assert torch.allclose(out["alpha"].cpu(), torch.ones(2), atol=1e-6)
+
+
+@pytest.mark.parametrize("name,nrows", [("C2", 10), ("C3", 8), ("C4", 6)])
+def test_full_size_configs_sampled_rows(name, nrows):
+    """Full-size workloads in the launch configuration the benchmark times; the checker recomputes a
+    seeded sample of rows one by one (all per-row outputs of those rows are compared)."""
+    cfg = W.CONFIGS[name]
+    inp = W.make_inputs(cfg, device="cuda")
+    rng = np.random.default_rng(cfg.seed)
+    rows = sorted(set([0, cfg.rows - 1] + rng.choice(cfg.rows, nrows, replace=False).tolist()))
+    t = _run_linear(cfg, inp, rows=rows, check_qtilde=False)
+    t.assert_ok(max_ambiguous_frac=0.2)
+    # properties that hold for every row at any size
+    rdk = _rdk()
+    idx = rdk.rdk_prepare_ids(inp["kept_ids"], cfg.N)
+    out = rdk.rdk_sample_and_verify(idx, rdk.binding.RDK_MODE_LINEAR, inp["target"], inp["drafter"], None,
+                                    inp["uniforms"], cfg.batch, cfg.positions)
+    torch.cuda.synchronize()
+    a, R, S = out["alpha"].double(), out["residual_mass"].double(), out["S"].double()
+    assert torch.all((a + R - 1).abs() < 2e-5)                      # Lemma 2.3: alpha = 1 - ||k||_1
+    assert torch.all((S - 1).abs() < 1e-3) and torch.all(a > 0) and torch.all(a <= 1 + 1e-6)
+    d = out["draft_token"].long()
+    assert torch.all((d >= 0) & (d < cfg.N))
+    ot = out["out_token"].long()
+    acc = out["accepted"].bool()
+    assert torch.all(ot[acc] == d[acc])
+    assert torch.all((out["accept_prob"] >= 0) & (out["accept_prob"] <= 1))
+    # acceptance frequency is consistent with the closed-form rate (binomial, 5 sigma)
+    mean_alpha = a.mean().item()
+    sigma = (a * (1 - a)).sum().sqrt().item() / cfg.rows
+    assert abs(acc.double().mean().item() - mean_alpha) < 5 * sigma + 1e-3
