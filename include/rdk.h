@@ -160,6 +160,27 @@ int rdk_redistribute_exact(const rdk_problem* problem, const void* drafter, cons
                            int32_t* status_word, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * rdk_redistribute_exact_static -- the paper has no counterpart; this is a packaging variant of
+ * rdk_redistribute_exact for callers that cannot allocate device memory: code running where
+ * cudaMalloc is off limits (inside a stream capture, in a latency-critical serving loop that must
+ * not touch the allocator, or in a host framework that owns all device memory and hands out only
+ * input and output buffers).  Same arguments and results as rdk_redistribute_exact, minus the
+ * workspace: the q' operand is staged in a fixed array of RDK_STATIC_SCRATCH_BYTES bytes that is
+ * part of the library image (each GPU that loads the library carries it until the process exits).
+ *   - Problems whose operand does not fit (rdk_exact_workspace_bytes(problem, layout) >
+ *     RDK_STATIC_SCRATCH_BYTES) are refused with RDK_ERR_WORKSPACE_TOO_SMALL; nothing is launched.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress);
+ *     make that first call outside any stream capture.  No call allocates or frees anything.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (the operand
+ *     is rewritten in full by every call), but two calls whose kernels overlap on the GPU, e.g. on
+ *     different streams, race on it: serialise them.
+ * ------------------------------------------------------------------------------------------- */
+#define RDK_STATIC_SCRATCH_BYTES (4u << 20)
+int rdk_redistribute_exact_static(const rdk_problem* problem, const void* drafter,
+                                  const rdk_affinity* M, float* w_out, float* S_out,
+                                  int32_t* status_word, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * rdk_redistribute_linear -- Eq. "rdk-taylor" written out to memory (the element-wise checkable
  * form of the linear path; rdk_sample_and_verify never stores this N-long vector).
  *   target      device [rows, N] target logits (p = softmax(target))

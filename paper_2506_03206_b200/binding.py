@@ -28,7 +28,7 @@ RDK_AFF_F32_ROWS, RDK_AFF_BF16_COLS = 0, 1
 EXPORTS = [
     "rdk_version", "rdk_status_string", "rdk_last_error", "rdk_kept_index_bytes", "rdk_prepare_ids",
     "rdk_build_affinity_workspace_bytes", "rdk_build_affinity", "rdk_exact_workspace_bytes",
-    "rdk_redistribute_exact", "rdk_redistribute_linear", "rdk_sample_and_verify",
+    "rdk_redistribute_exact", "rdk_redistribute_exact_static", "rdk_redistribute_linear", "rdk_sample_and_verify",
     "rdk_sample_and_verify_host",
 ]
 
@@ -87,6 +87,9 @@ def lib() -> C.CDLL:
         L.rdk_redistribute_exact.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.POINTER(rdk_affinity),
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p,
                                              C.c_void_p]
+        L.rdk_redistribute_exact_static.restype = C.c_int
+        L.rdk_redistribute_exact_static.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.POINTER(rdk_affinity),
+                                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.rdk_redistribute_linear.restype = C.c_int
         L.rdk_redistribute_linear.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.c_void_p, C.c_void_p,
                                               C.c_void_p, C.c_void_p, C.c_void_p]
@@ -221,6 +224,23 @@ def rdk_redistribute_exact(index: KeptIndex, drafter: torch.Tensor, M: Dict[str,
                                         S.data_ptr(), ws.data_ptr(), ws.numel(), _ptr(status_word), _stream()),
            "rdk_redistribute_exact")
     return w_out, S, ws
+
+
+RDK_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def rdk_redistribute_exact_static(index: KeptIndex, drafter: torch.Tensor, M: Dict[str, object], batch: int,
+                                  positions: int, w_out: torch.Tensor, S_out: torch.Tensor,
+                                  drafter_kind: int = RDK_LOGITS, status_word: Optional[torch.Tensor] = None) -> None:
+    """rdk_redistribute_exact without a workspace argument: the library stages the q' operand in its
+    own fixed device array, so this call (and this wrapper) allocates nothing -- the caller passes
+    the output tensors in.  Meant for callers that must not touch the device allocator."""
+    _rows2d(drafter, "drafter")
+    pb = make_problem(index, None, drafter, batch, positions, drafter_kind)
+    a = _aff_struct(M)
+    _check(lib().rdk_redistribute_exact_static(C.byref(pb), drafter.data_ptr(), C.byref(a), w_out.data_ptr(),
+                                               S_out.data_ptr(), _ptr(status_word), _stream()),
+           "rdk_redistribute_exact_static")
 
 
 def rdk_redistribute_linear(index: KeptIndex, target: torch.Tensor, drafter: torch.Tensor, batch: int,

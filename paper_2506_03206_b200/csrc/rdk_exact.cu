@@ -209,3 +209,57 @@ extern "C" int rdk_redistribute_exact(const rdk_problem* problem, const void* dr
     }
     return RDK_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Variant of rdk_redistribute_exact whose q' operand lives in a fixed device array instead of a
+// caller-supplied workspace, for callers that are not able to allocate device memory.
+// ------------------------------------------------------------------------------------------------
+#include <mutex>
+
+static __device__ __align__(256) unsigned char g_exact_static_scratch[RDK_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" int rdk_redistribute_exact_static(const rdk_problem* problem, const void* drafter,
+                                             const rdk_affinity* M, float* w_out, float* S_out,
+                                             int32_t* status_word, void* stream) {
+    if (!problem || !M) {
+        set_error("rdk_redistribute_exact_static: null pointer");
+        return RDK_ERR_INVALID_ARG;
+    }
+    const size_t need = rdk_exact_workspace_bytes(problem, M->layout);
+    if (need == 0) {
+        set_error("rdk_redistribute_exact_static: bad sizes or affinity layout");
+        return RDK_ERR_INVALID_ARG;
+    }
+    if (need > (size_t)RDK_STATIC_SCRATCH_BYTES) {
+        set_error("rdk_redistribute_exact_static: the q' operand needs %zu bytes but the built-in scratch array holds "
+                  "%zu; use rdk_redistribute_exact with your own workspace", need, (size_t)RDK_STATIC_SCRATCH_BYTES);
+        return RDK_ERR_WORKSPACE_TOO_SMALL;
+    }
+    int dev = 0;
+    RDK_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) {
+        set_error("rdk_redistribute_exact_static: device ordinal %d not supported", dev);
+        return RDK_ERR_UNSUPPORTED;
+    }
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_ptr[dev]) {
+            // The array's name is only a host-side handle; the kernels need its device address.
+            void* p = nullptr;
+            RDK_CUDA(cudaGetSymbolAddress(&p, g_exact_static_scratch));
+            g_scratch_ptr[dev] = p;
+        }
+        scratch = g_scratch_ptr[dev];
+    }
+    // Every element of the operand that the contraction reads is written first by the operand
+    // kernel (padding columns included), so nothing left over from an earlier call is ever used.
+    return rdk_redistribute_exact(problem, drafter, M, w_out, S_out, scratch, (size_t)RDK_STATIC_SCRATCH_BYTES,
+                                  status_word, stream);
+}
