@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
 NCU_TRAFFIC = {"sources_sha256": None, "bytes_per_launch": None}
-KERNEL_SOURCES = ("rdk_row.cu", "rdk_common.cuh")
+KERNEL_SOURCES = ("rdk_row_cluster.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 
 def _kernel_sources_hash() -> str:
@@ -212,11 +212,13 @@ def run_ours(args):
     index = B.rdk_prepare_ids(sets[0]["kept_ids"], cfg.N)
     outs = [B.alloc_outputs(rows, cfg.batch, trials, dev) for _ in range(N_BUFFER_SETS)]
     outs_nolen = [{k: v for k, v in o.items() if k != "accepted_len"} for o in outs]
+    pb = B.make_problem(index, sets[0]["target"], sets[0]["drafter"], cfg.batch, cfg.positions)
+    ws = B.sample_workspace(pb, B.RDK_MODE_LINEAR, trials, dev)
 
     def step(i, out_list=outs):
         s = sets[i % N_BUFFER_SETS]
         B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, s["target"], s["drafter"], None, s["uniforms"],
-                                cfg.batch, cfg.positions, out=out_list[i % N_BUFFER_SETS])
+                                cfg.batch, cfg.positions, out=out_list[i % N_BUFFER_SETS], ws=ws)
 
     def barrier():
         torch.cuda.synchronize()
@@ -257,8 +259,8 @@ def run_ours(args):
     for s in sets[:2]:
         host_sets.append({k: s[k].cpu().pin_memory() for k in ("target", "drafter", "uniforms")})
     stage = {"target": torch.empty_like(sets[0]["target"]), "drafter": torch.empty_like(sets[0]["drafter"]),
-             "uniforms": torch.empty_like(sets[0]["uniforms"])}
-    host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in outs[0].items()}
+             "uniforms": torch.empty_like(sets[0]["uniforms"]), "ws": ws}
+    host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in outs[0].items() if not k.startswith("_")}
 
     def e2e_step(i):
         h = host_sets[i % len(host_sets)]

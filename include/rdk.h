@@ -204,11 +204,18 @@ int rdk_redistribute_linear(const rdk_problem* problem, const void* target, cons
  *   uniforms   device float [rows, trials, 4] in [0, 1)
  *   trials     >= 1 independent draws per row (each uses its own 4 uniforms)
  *   out        see rdk_outputs
+ *   ws         device workspace of rdk_sample_workspace_bytes(problem, mode, trials) bytes, 256-byte
+ *              aligned (may be NULL when that size is 0).  It holds, between the two kernels of
+ *              the linear path, one record of 1088 bytes per row (row scalars and per-segment sums
+ *              of w, min(p, q~), max(0, p - q~), p) and one counter per (sequence, trial).
+ * Arithmetic of the linear mode: fp32; for N >= 4096 the quotient 1 / (N + p_j) is expanded as
+ * (1/N)(1 - x + x^2), x = p_j / N <= 2^-12 (relative truncation below 2^-36), otherwise divided.
  * ------------------------------------------------------------------------------------------- */
+size_t rdk_sample_workspace_bytes(const rdk_problem* problem, int32_t mode, int32_t trials);
 int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* target,
                           const void* drafter, const float* w, int64_t w_row_stride,
                           const float* uniforms, int32_t trials, const rdk_outputs* out,
-                          void* stream);
+                          void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * rdk_sample_and_verify_host -- the same step (linear mode) for callers whose logits live in HOST
@@ -218,13 +225,14 @@ int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* 
  *   problem->kept_index, staging buffers: device.   *_host: host.
  *   stage_target [rows * N], stage_drafter [rows * n] of the problem's dtypes, stage_uniforms
  *   float [rows * trials * 4], dev_out: device outputs as in rdk_outputs (members that are NULL
- *   are skipped, also in host_out); host_out: host arrays of the same shapes.
+ *   are skipped, also in host_out); host_out: host arrays of the same shapes; ws as in
+ *   rdk_sample_and_verify.
  * ------------------------------------------------------------------------------------------- */
 int rdk_sample_and_verify_host(const rdk_problem* problem, const void* target_host,
                                const void* drafter_host, const float* uniforms_host,
                                int32_t trials, void* stage_target, void* stage_drafter,
                                float* stage_uniforms, const rdk_outputs* dev_out,
-                               const rdk_outputs* host_out, void* stream);
+                               const rdk_outputs* host_out, void* ws, size_t ws_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -28,7 +28,8 @@ RDK_AFF_F32_ROWS, RDK_AFF_BF16_COLS = 0, 1
 EXPORTS = [
     "rdk_version", "rdk_status_string", "rdk_last_error", "rdk_kept_index_bytes", "rdk_prepare_ids",
     "rdk_build_affinity_workspace_bytes", "rdk_build_affinity", "rdk_exact_workspace_bytes",
-    "rdk_redistribute_exact", "rdk_redistribute_exact_static", "rdk_redistribute_linear", "rdk_sample_and_verify",
+    "rdk_redistribute_exact", "rdk_redistribute_exact_static", "rdk_redistribute_linear",
+    "rdk_sample_workspace_bytes", "rdk_sample_and_verify",
     "rdk_sample_and_verify_host",
 ]
 
@@ -96,11 +97,14 @@ def lib() -> C.CDLL:
         L.rdk_sample_and_verify.restype = C.c_int
         L.rdk_sample_and_verify.argtypes = [C.POINTER(rdk_problem), C.c_int32, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_int64, C.c_void_p, C.c_int32,
-                                            C.POINTER(rdk_outputs), C.c_void_p]
+                                            C.POINTER(rdk_outputs), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.rdk_sample_workspace_bytes.restype = C.c_size_t
+        L.rdk_sample_workspace_bytes.argtypes = [C.POINTER(rdk_problem), C.c_int32, C.c_int32]
         L.rdk_sample_and_verify_host.restype = C.c_int
         L.rdk_sample_and_verify_host.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.c_void_p, C.c_void_p,
                                                  C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
-                                                 C.POINTER(rdk_outputs), C.POINTER(rdk_outputs), C.c_void_p]
+                                                 C.POINTER(rdk_outputs), C.POINTER(rdk_outputs), C.c_void_p,
+                                                 C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -276,15 +280,21 @@ def alloc_outputs(rows: int, batch: int, trials: int, device) -> Dict[str, torch
 def outputs_struct(out: Dict[str, torch.Tensor]) -> rdk_outputs:
     o = rdk_outputs()
     for name, _ in rdk_outputs._fields_:
-        setattr(o, name, _ptr(out.get(name)))
+        setattr(o, name, _ptr(out.get(name)))   # absent members stay NULL
     return o
+
+
+def sample_workspace(pb: rdk_problem, mode: int, trials: int, device) -> torch.Tensor:
+    nbytes = lib().rdk_sample_workspace_bytes(C.byref(pb), mode, trials)
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
 
 
 def rdk_sample_and_verify(index: KeptIndex, mode: int, target: torch.Tensor,
                           drafter: Optional[torch.Tensor], w: Optional[torch.Tensor],
                           uniforms: torch.Tensor, batch: int, positions: int,
                           drafter_kind: int = RDK_LOGITS,
-                          out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+                          out: Optional[Dict[str, torch.Tensor]] = None,
+                          ws: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
     _rows2d(target, "target")
     rows = batch * positions
     if uniforms.dtype != torch.float32 or not uniforms.is_contiguous() or uniforms.numel() % (rows * 4):
@@ -294,9 +304,12 @@ def rdk_sample_and_verify(index: KeptIndex, mode: int, target: torch.Tensor,
     if out is None:
         out = alloc_outputs(rows, batch, trials, target.device)
     o = outputs_struct(out)
+    if ws is None:
+        ws = sample_workspace(pb, mode, trials, target.device)
     _check(lib().rdk_sample_and_verify(C.byref(pb), mode, target.data_ptr(), _ptr(drafter), _ptr(w),
                                        0 if w is None else w.stride(0), uniforms.data_ptr(), trials,
-                                       C.byref(o), _stream()), "rdk_sample_and_verify")
+                                       C.byref(o), ws.data_ptr(), ws.numel(), _stream()), "rdk_sample_and_verify")
+    out["_ws"] = ws        # keep the workspace alive until the stream has consumed it
     return out
 
 
@@ -304,6 +317,7 @@ def rdk_sample_and_verify_host(index: KeptIndex, target_host: torch.Tensor, draf
                                uniforms_host: torch.Tensor, batch: int, positions: int, stage: Dict[str, torch.Tensor],
                                dev_out: Dict[str, torch.Tensor], host_out: Dict[str, torch.Tensor],
                                drafter_kind: int = RDK_LOGITS) -> Dict[str, torch.Tensor]:
+    """`stage` holds the device staging tensors "target", "drafter", "uniforms" and the workspace "ws"."""
     rows = batch * positions
     trials = uniforms_host.numel() // (rows * 4)
     pb = make_problem(index, stage["target"], stage["drafter"], batch, positions, drafter_kind)
@@ -311,7 +325,8 @@ def rdk_sample_and_verify_host(index: KeptIndex, target_host: torch.Tensor, draf
     _check(lib().rdk_sample_and_verify_host(C.byref(pb), target_host.data_ptr(), drafter_host.data_ptr(),
                                             uniforms_host.data_ptr(), trials, stage["target"].data_ptr(),
                                             stage["drafter"].data_ptr(), stage["uniforms"].data_ptr(),
-                                            C.byref(od), C.byref(oh), _stream()), "rdk_sample_and_verify_host")
+                                            C.byref(od), C.byref(oh), stage["ws"].data_ptr(), stage["ws"].numel(),
+                                            _stream()), "rdk_sample_and_verify_host")
     return host_out
 
 

@@ -389,7 +389,7 @@ static bool force_generic_kernel() {
 static int run_rows(const rdk_problem* pb, int mode, const void* target, const void* drafter,
                     const float* w, long long w_stride, const float* uniforms, int trials,
                     const rdk_outputs* out, float* qtilde, float* theta_out, float* S_out,
-                    cudaStream_t s) {
+                    void* ws, size_t ws_bytes, cudaStream_t s) {
     RowParams P{};
     P.N = pb->N; P.n = pb->n; P.rows = pb->batch * pb->positions; P.trials = trials;
     P.target = target; P.target_stride = pb->target_row_stride ? pb->target_row_stride : pb->N;
@@ -411,8 +411,12 @@ static int run_rows(const rdk_problem* pb, int mode, const void* target, const v
     P.num_tiles = (pb->N + kTile - 1) / kTile;
     const size_t smem = (size_t)P.num_tiles * kRowWarps * 24;
     cudaError_t e = cudaErrorNotSupported;
-    if (mode == RDK_MODE_LINEAR && trials > 0 && !force_generic_kernel())
-        e = launch_cluster_linear(P, pb->target_dtype, pb->drafter_dtype, pb->drafter_kind, s);
+    P.positions = pb->positions;
+    P.accepted_len = out ? out->accepted_len : nullptr;
+    if (mode == RDK_MODE_LINEAR && trials > 0 && !force_generic_kernel()) {
+        e = launch_cluster_linear(P, pb->target_dtype, pb->drafter_dtype, pb->drafter_kind, pb->batch, ws, ws_bytes, s);
+        if (e == cudaSuccess) return RDK_OK;          // the draw kernel also wrote accepted_len
+    }
     if (e == cudaErrorNotSupported)
         e = (mode == RDK_MODE_LINEAR)
             ? launch_types<RDK_MODE_LINEAR>(P, pb->target_dtype, pb->drafter_dtype, pb->drafter_kind, smem, s)
@@ -440,13 +444,20 @@ extern "C" int rdk_redistribute_linear(const rdk_problem* problem, const void* t
     st = check_arch();
     if (st != RDK_OK) return st;
     return run_rows(problem, RDK_MODE_LINEAR, target, drafter, nullptr, 0, nullptr, 0, nullptr,
-                    qtilde_out, theta_out, S_out, static_cast<cudaStream_t>(stream));
+                    qtilde_out, theta_out, S_out, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t rdk_sample_workspace_bytes(const rdk_problem* problem, int32_t mode, int32_t trials) {
+    if (!problem || mode != RDK_MODE_LINEAR || trials < 1 || problem->batch < 1 || problem->positions < 1) return 0;
+    const long long rows = (long long)problem->batch * problem->positions;
+    if (rows > 0x7fffffffLL) return 0;
+    return cluster_workspace_bytes((int)rows, problem->batch, trials);
 }
 
 extern "C" int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* target,
                                      const void* drafter, const float* w, int64_t w_row_stride,
                                      const float* uniforms, int32_t trials, const rdk_outputs* out,
-                                     void* stream) {
+                                     void* ws, size_t ws_bytes, void* stream) {
     if (mode != RDK_MODE_LINEAR && mode != RDK_MODE_PRECOMPUTED_W) {
         set_error("rdk_sample_and_verify: unknown mode %d", mode);
         return RDK_ERR_INVALID_ARG;
@@ -469,17 +480,22 @@ extern "C" int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, c
         set_error("rdk_sample_and_verify: accepted_len needs the accepted output");
         return RDK_ERR_INVALID_ARG;
     }
+    const size_t need = rdk_sample_workspace_bytes(problem, mode, trials);
+    if (need > 0 && (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u))) {
+        set_error("rdk_sample_and_verify: workspace of %zu bytes (256-byte aligned) needed, %zu given", need, ws ? ws_bytes : (size_t)0);
+        return RDK_ERR_WORKSPACE_TOO_SMALL;
+    }
     st = check_arch();
     if (st != RDK_OK) return st;
     return run_rows(problem, mode, target, drafter, w, w_row_stride, uniforms, trials, out, nullptr,
-                    nullptr, nullptr, static_cast<cudaStream_t>(stream));
+                    nullptr, nullptr, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int rdk_sample_and_verify_host(const rdk_problem* problem, const void* target_host,
                                           const void* drafter_host, const float* uniforms_host,
                                           int32_t trials, void* stage_target, void* stage_drafter,
                                           float* stage_uniforms, const rdk_outputs* dev_out,
-                                          const rdk_outputs* host_out, void* stream) {
+                                          const rdk_outputs* host_out, void* ws, size_t ws_bytes, void* stream) {
     int st = validate_problem(problem, "rdk_sample_and_verify_host", true);
     if (st != RDK_OK) return st;
     if (!target_host || !drafter_host || !uniforms_host || !stage_target || !stage_drafter ||
@@ -501,7 +517,7 @@ extern "C" int rdk_sample_and_verify_host(const rdk_problem* problem, const void
     RDK_CUDA(cudaMemcpyAsync(stage_drafter, drafter_host, rows * problem->n * yb, cudaMemcpyHostToDevice, s));
     RDK_CUDA(cudaMemcpyAsync(stage_uniforms, uniforms_host, rows * trials * 4 * sizeof(float), cudaMemcpyHostToDevice, s));
     st = rdk_sample_and_verify(problem, RDK_MODE_LINEAR, stage_target, stage_drafter, nullptr, 0,
-                               stage_uniforms, trials, dev_out, stream);
+                               stage_uniforms, trials, dev_out, ws, ws_bytes, stream);
     if (st != RDK_OK) return st;
     const size_t rt = rows * trials;
 #define RDK_BACK(member, count, type)                                                             \

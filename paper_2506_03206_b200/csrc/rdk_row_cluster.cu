@@ -1,8 +1,14 @@
-// Cluster kernel for the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8).
+// Two-kernel form of the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8) for N >= 4096.
 //
-// One thread-block cluster of C CTAs takes one row.  CTA c keeps its slice of the target logits
-// resident in shared memory (one TMA bulk copy), so the row is read from HBM exactly once; the
-// C partial results are exchanged through distributed shared memory.
+// Kernel 1 (rdk_stream_kernel): one thread-block cluster of C CTAs per row.  CTA c brings its slice
+// of the target logits into shared memory with TMA bulk copies, so the row is read from HBM exactly
+// once; the C partial results are exchanged once through distributed shared memory.  It leaves a
+// small record per row in the workspace: the row's scalars and, for each of the C*8 contiguous
+// token segments, the sums of w, of min(p, q~), of max(0, p - q~) and of p.
+// Kernel 2 (rdk_draw_kernel): one CTA per (row, trial) turns the record into draws: it locates the
+// segment by prefix sums over the record, re-reads that one segment (about N/64 tokens, usually
+// still in L2), picks the token, runs the rejection test and the residual draw, and counts the
+// accepted prefix of each sequence.
 //
 // Arithmetic, with p = softmax(z), q' = TLI(softmax(y)), x_j = p_j / N:
 //   w_j = (N q'_j + theta p_j) / (N + p_j) = (q'_j + theta x_j) / (1 + x_j)
@@ -10,10 +16,9 @@
 // * A token the drafter does not keep has q'_j = 0, hence w_j / S < p_j: its share of
 //   alpha = sum min(p, q~) is w_j / S and its residual is p_j - w_j / S.  All such tokens enter only
 //   through sum p_j and sum p_j^2 per segment, which come out of the soft-max sweep itself.
-// * The n kept tokens are evaluated one by one (cached in shared memory as (p_j, w_j)).
+// * The n kept tokens are evaluated one by one from values cached in shared memory.
 // * S = sum_j w_j = 1 + (sum_j q'_j p_j^2 - theta sum_j p_j^2) / N^2 + O(N^-3), because
 //   sum q' = 1 and sum q'_j p_j = theta cancel the first-order terms.
-// The kernel is used for N >= 4096 only, where the truncated series is below fp32 resolution.
 #include <cooperative_groups.h>
 
 #include "rdk_row.cuh"
@@ -22,29 +27,24 @@ namespace cg = cooperative_groups;
 
 namespace rdk {
 
-constexpr int kCT = 256;             // threads per CTA
-constexpr int kCW = kCT / 32;        // warps per CTA; each owns a contiguous token range = one CDF segment
+constexpr int kCT = 256;             // threads per CTA of kernel 1
+constexpr int kCW = kCT / 32;        // warps per CTA; each owns a contiguous token range = one segment
 constexpr int kMaxC = 8;             // portable cluster size
 constexpr int kMaxSeg = kMaxC * kCW;
-constexpr int kTrialBatch = kCW;     // trials handled between two cluster exchanges (one per warp)
 constexpr int kMinClusterN = 4096;
 constexpr unsigned kSpinLimit = 1u << 22;
+constexpr int kDT = 512;             // threads per CTA of kernel 2: 8 warps for the draft, 8 for the residual
+constexpr int kMaxChunks = 128;      // 256-token chunks per segment (N <= 2^21)
 
-struct Pub1 {    // per-CTA partials, published before the first exchange
+// record layout (floats): 16 scalars, then 4 per segment
+enum { kRecOffg = 0, kRecInvZp, kRecYoffg, kRecInvZq, kRecTheta, kRecInvN, kRecInvS, kRecS };
+
+struct Pub1 {    // per-CTA partials, published before the exchange
     float m, my;
     float E1[kCW], E2[kCW], K1[kCW], K2[kCW], Zq[kCW], th[kCW], q2[kCW];
 };
-struct Pub2 { float Kw[kCW], ak[kCW]; };
-struct Pub3 { int d[kTrialBatch]; float pd[kTrialBatch], wd[kTrialBatch]; };
 
-struct CCtx {
-    const void* zbuf; float2* cache; int cap;
-    const uint32_t* mask; const int32_t* rank; const int32_t* slot;
-    const void* yrow;
-    int N, j0, r0;
-    bool identity;
-    float offg, inv_zp, yoffg, inv_zq, theta, inv_n, inv_s;
-};
+struct Scal { float offg, inv_zp, yoffg, inv_zq, theta, inv_n, inv_s; };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -72,106 +72,31 @@ __device__ __forceinline__ int rank_at(const RowParams& P, int j, int n_valid) {
 }
 
 // w_j for given p_j and q'_j:  (q' + theta x) (1 - x + x^2),  x = p / N
-__device__ __forceinline__ float taylor_w(const CCtx& c, float p, float qp) {
+__device__ __forceinline__ float taylor_w(const Scal& c, float p, float qp) {
     const float x = p * c.inv_n;
     return fmaf(c.theta, x, qp) * fmaf(x, x - 1.f, 1.f);
 }
 
-// p and w of the 8 tokens at local index jl (a multiple of 8) of this CTA's slice
-template <typename TZ, typename TY, int KIND>
-__device__ __forceinline__ void chunk_pw(const CCtx& c, int jl, float (&p)[kVec], float (&w)[kVec]) {
-    float z[kVec];
-    lds8<TZ>(static_cast<const TZ*>(c.zbuf), jl, z);
-#pragma unroll
-    for (int k = 0; k < kVec; ++k) {
-        p[k] = ex2(fmaf(z[k], kLog2e, c.offg)) * c.inv_zp;
-        w[k] = taylor_w(c, p[k], 0.f);
-    }
-    const int jg = c.j0 + jl;
-    if (jg >= c.N) return;
-    const uint32_t word = __ldg(c.mask + (jg >> 5));
-    const int sh = jg & 31;
-    const uint32_t mb = (word >> sh) & 0xffu;
-    if (!mb) return;
-    int r = __ldg(c.rank + (jg >> 5)) + __popc(word & ((1u << sh) - 1u));
-#pragma unroll
-    for (int k = 0; k < kVec; ++k) {
-        if (mb & (1u << k)) {
-            const int il = r - c.r0;
-            if (il < c.cap) {
-                const float2 v = c.cache[il];
-                p[k] = v.x; w[k] = v.y;
-            } else {
-                const int i = c.identity ? r : __ldg(c.slot + r);
-                const float y = to_float<TY>(static_cast<const TY*>(c.yrow)[i]);
-                const float qp = (KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, c.yoffg)) : y) * c.inv_zq;
-                w[k] = taylor_w(c, p[k], qp);
-            }
-            ++r;
-        }
-    }
+__device__ __forceinline__ bool index_matches(const RowParams& P) {
+    return P.header[kHdrMagic] == kIdxMagic && P.header[kHdrN] == P.N && P.header[kHdrn] == P.n;
 }
 
-enum { kPickW = 0, kPickR = 1, kPickP = 2 };
-
-// Inverse-CDF pick inside the local token range [a, b) of this CTA's slice (one warp):
-// the first token whose running sum of weights exceeds rem; if rounding leaves none, the last
-// positive one.  Returns the local token index (or -1 if every weight is zero) and its p, w.
-template <typename TZ, typename TY, int KIND, int WHAT>
-__device__ __forceinline__ int pick_in_range(const CCtx& c, int a, int b, float rem, int lane, float& p_sel, float& w_sel) {
-    float cum = 0.f;
-    int last_cs = -1;
-    for (int pass = 0; pass < 2; ++pass) {
-        for (int cs = (pass == 0 ? a : last_cs); cs < b; cs += kSeg) {
-            const int jl = cs + lane * kVec;
-            float p[kVec], w[kVec], x[kVec];
-#pragma unroll
-            for (int k = 0; k < kVec; ++k) { p[k] = 0.f; w[k] = 0.f; }
-            if (jl < b) chunk_pw<TZ, TY, KIND>(c, jl, p, w);
-            float sum = 0.f;
-#pragma unroll
-            for (int k = 0; k < kVec; ++k) {
-                x[k] = WHAT == kPickW ? w[k] : (WHAT == kPickR ? fmaxf(0.f, p[k] - w[k] * c.inv_s) : p[k]);
-                sum += x[k];
-            }
-            sum = warp_sum(sum);
-            if (sum > 0.f) {
-                const bool take = pass == 1 || cum + sum > rem;
-                if (take) {
-                    const int sel = pick_in_segment(x, pass == 1 ? INFINITY : rem - cum, lane);
-                    float ps = 0.f, ws = 0.f;
-#pragma unroll
-                    for (int k = 0; k < kVec; ++k) if (k == (sel & (kVec - 1))) { ps = p[k]; ws = w[k]; }
-                    p_sel = __shfl_sync(0xffffffffu, ps, sel / kVec);
-                    w_sel = __shfl_sync(0xffffffffu, ws, sel / kVec);
-                    return cs + sel;
-                }
-                last_cs = cs;
-                cum += sum;
-            }
-            if (pass == 1) break;
-        }
-        if (last_cs < 0) break;
-    }
-    p_sel = 0.f; w_sel = 0.f;
-    return -1;
-}
-
+// ------------------------------------------------------------------------------------------------
+// kernel 1
+// ------------------------------------------------------------------------------------------------
 template <typename TZ, typename TY, int KIND>
 __global__ void __launch_bounds__(kCT)
-rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) {
+rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap) {
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(128) unsigned char dsm[];
     TZ* zbuf = reinterpret_cast<TZ*>(dsm);
     float2* cache = reinterpret_cast<float2*>(dsm + (((size_t)Ls * sizeof(TZ) + 127) & ~size_t(127)));
 
     __shared__ Pub1 pub1;
-    __shared__ Pub2 pub2;
-    __shared__ Pub3 pub3;
-    __shared__ float segA[kMaxSeg], segP[kMaxSeg];
-    __shared__ double cdfW[kMaxSeg], cdfR[kMaxSeg], cdfP[kMaxSeg];
-    __shared__ float bc[16];
+    __shared__ float segA[kCW], segP[kCW];
+    __shared__ float bc[12];
     __shared__ float redm[kCW], redy[kCW];
+    __shared__ int rk[kCW + 1];
     __shared__ __align__(8) unsigned long long bar;
     __shared__ int fail;
 
@@ -179,18 +104,16 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
     const int crank = (int)cluster.block_rank();
     const int row = blockIdx.x / C;
 
-    {   // the kept-id index must belong to this problem (same decision in every CTA)
-        const bool ok = P.header[kHdrMagic] == kIdxMagic && P.header[kHdrN] == P.N && P.header[kHdrn] == P.n;
-        if (!ok) {
-            if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
-            return;
-        }
+    if (!index_matches(P)) {   // same decision in every CTA of the grid; nothing is in flight yet
+        if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
+        return;
     }
     const bool identity = P.header[kHdrIdentity] != 0;
     const int n_valid = P.header[kHdrValid];
 
     const int j0 = crank * Ls;
     const int len = max(0, min(P.N - j0, Ls));
+    const int Lw = Ls / kCW;
     const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
     const TY* yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
 
@@ -211,17 +134,20 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
             }
         }
     }
+    if (tid <= kCW) rk[tid] = rank_at(P, min(P.N, j0 + tid * Lw), n_valid);   // rank at the warp range borders
     for (int idx = len8 + tid; idx < Ls; idx += kCT) zbuf[idx] = idx < len ? zrow[j0 + idx] : neg_inf<TZ>();
     __syncthreads();
 
-    // ---- drafter slice: raw values into the cache, running max ----------------------------------
-    const int r0 = rank_at(P, j0, n_valid), r1 = rank_at(P, min(P.N, j0 + Ls), n_valid);
-    const int kc = r1 - r0;
+    // ---- drafter slice: (local token index, raw value) into the cache, running max ---------------
+    const int r0 = rk[0];
+    const int kc = rk[kCW] - r0;
     float my_t = -INFINITY;
+#pragma unroll 4
     for (int il = tid; il < kc; il += kCT) {
         const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
         const float y = to_float<TY>(yrow[i]);
-        if (il < cap) cache[il].y = y;
+        const int jl = __ldg(P.ids + i) - j0;
+        if (il < cap) cache[il] = make_float2(__int_as_float(jl), y);
         if (KIND == RDK_LOGITS) my_t = fmaxf(my_t, y);
     }
 
@@ -236,7 +162,6 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
     }
 
     // ---- slice maximum of z -------------------------------------------------------------------
-    const int Lw = Ls / kCW;
     const int wa = warp * Lw, wb = wa + Lw;
     float mz_t = -INFINITY;
     for (int cs = wa; cs < wb; cs += kSeg) {
@@ -276,13 +201,19 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
         }
     }
     // ---- kept tokens of the warp's range: e_z, e_y, their sums ------------------------------------
-    const int rw0 = rank_at(P, min(P.N, j0 + wa), n_valid) - r0, rw1 = rank_at(P, min(P.N, j0 + wb), n_valid) - r0;
+    const int rw0 = rk[warp] - r0, rw1 = rk[warp + 1] - r0;
     float K1 = 0.f, K2 = 0.f, Zq = 0.f, th = 0.f, q2 = 0.f;
+#pragma unroll 2
     for (int il = rw0 + lane; il < rw1; il += 32) {
-        const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
-        const int jl = __ldg(P.ids + i) - j0;
+        int jl;
+        float y;
+        if (il < cap) { const float2 v = cache[il]; jl = __float_as_int(v.x); y = v.y; }
+        else {
+            const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
+            jl = __ldg(P.ids + i) - j0;
+            y = to_float<TY>(yrow[i]);
+        }
         const float ez = ex2(fmaf(to_float<TZ>(zbuf[jl]), kLog2e, zoff_c));
-        const float y = il < cap ? cache[il].y : to_float<TY>(yrow[i]);
         const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
         K1 += ez;
         K2 = fmaf(ez, ez, K2);
@@ -298,7 +229,7 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
         pub1.Zq[warp] = Zq; pub1.th[warp] = th; pub1.q2[warp] = q2;
     }
     if (tid == 0) { pub1.m = m_c; pub1.my = my_c; }
-    cluster.sync();                                                            // exchange 1
+    cluster.sync();                                                            // the one exchange
 
     // ---- combine the C partials (warp 0 of every CTA, same order everywhere) ----------------------
     const int nseg = C * kCW;
@@ -336,11 +267,11 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
 #pragma unroll
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
-            if (s < nseg) {
+            if (s < nseg && s / kCW == crank) {
                 const float Po = fmaxf(0.f, e1[it] - k1[it]) * inv_zp;
                 const float P2o = fmaxf(0.f, e2[it] - k2[it]) * inv_zp * inv_zp;
-                segP[s] = e1[it] * inv_zp;
-                segA[s] = inv_n * (Po - inv_n * P2o);       // sum over not-kept tokens of p / (N + p)
+                segP[s % kCW] = e1[it] * inv_zp;
+                segA[s % kCW] = inv_n * (Po - inv_n * P2o);       // sum over not-kept tokens of p / (N + p)
             }
         }
         const float f_me = __shfl_sync(0xffffffffu, f_l, crank), g_me = __shfl_sync(0xffffffffu, g_l, crank);
@@ -350,15 +281,15 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
             bc[9] = S;
         }
     }
+    cluster.barrier_arrive();          // this thread reads no remote shared memory from here on
     __syncthreads();
-    CCtx c;
-    c.zbuf = zbuf; c.cache = cache; c.cap = cap; c.mask = P.mask; c.rank = P.rank; c.slot = P.slot; c.yrow = yrow;
-    c.N = P.N; c.j0 = j0; c.r0 = r0; c.identity = identity;
+    Scal c;
     c.offg = bc[0]; c.inv_zp = bc[1]; c.yoffg = bc[2]; c.inv_zq = bc[3]; c.theta = bc[4]; c.inv_n = bc[5]; c.inv_s = bc[6];
     const float fz = bc[7], fy = bc[8];
 
     // ---- kept tokens again: p, w, min(p, q~) ---------------------------------------------------
     float Kw = 0.f, ak = 0.f;
+#pragma unroll 2
     for (int il = rw0 + lane; il < rw1; il += 32) {
         float ez, ey;
         if (il < cap) { const float2 v = cache[il]; ez = v.x; ey = v.y; }
@@ -372,172 +303,291 @@ rdk_cluster_kernel(const RowParams P, const int C, const int Ls, const int cap) 
         const float w = taylor_w(c, p, qp);
         Kw += w;
         ak += fminf(p, w * c.inv_s);
-        if (il < cap) cache[il] = make_float2(p, w);
     }
     Kw = warp_sum(Kw); ak = warp_sum(ak);
-    if (lane == 0) { pub2.Kw[warp] = Kw; pub2.ak[warp] = ak; }
-    cluster.sync();                                                            // exchange 2
 
-    // ---- per-segment totals and their prefix sums (fp64), row outputs -----------------------------
-    if (warp == 0) {
-        double sw[2], sr[2], sp[2];
+    // ---- the row's record ---------------------------------------------------------------------
+    float* rec = P.rec + (long long)row * kRecFloats;
+    if (lane == 0) {
+        const float oov = c.theta * segA[warp];
+        const float w_s = oov + Kw;
+        const float a_s = oov * c.inv_s + ak;
+        reinterpret_cast<float4*>(rec + 16)[crank * kCW + warp] = make_float4(w_s, a_s, fmaxf(0.f, segP[warp] - a_s), segP[warp]);
+    }
+    if (crank == 0) {
+        if (tid < 8) rec[tid] = tid < 7 ? bc[tid] : bc[9];
+        if (P.counters && row % P.positions == 0)
+            for (int t = tid; t < P.trials; t += kCT) P.counters[(row / P.positions) * P.trials + t] = 0;
+    }
+    if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
+    cluster.barrier_wait();            // remote shared memory must outlive its readers
+}
+
+// ------------------------------------------------------------------------------------------------
+// kernel 2
+// ------------------------------------------------------------------------------------------------
+struct DrawCtx {
+    const void* zrow; const void* yrow; bool zvec;
+    const uint32_t* mask; const int32_t* rank; const int32_t* slot;
+    int N; bool identity;
+    Scal c;
+};
+
+// p and w of the 8 tokens starting at global token jb (a multiple of 8)
+template <typename TZ, typename TY, int KIND>
+__device__ __forceinline__ void draw_pw(const DrawCtx& d, int jb, float (&p)[kVec], float (&w)[kVec]) {
+    float z[kVec];
+    load8<TZ>(static_cast<const TZ*>(d.zrow), jb, d.N, d.zvec, -INFINITY, z);
+    const uint32_t word = __ldg(d.mask + (jb >> 5));
+    const int sh = jb & 31;
+    const uint32_t mb = (word >> sh) & 0xffu;
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) {
+        p[k] = ex2(fmaf(z[k], kLog2e, d.c.offg)) * d.c.inv_zp;
+        w[k] = taylor_w(d.c, p[k], 0.f);
+    }
+    if (!mb) return;
+    int r = __ldg(d.rank + (jb >> 5)) + __popc(word & ((1u << sh) - 1u));
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) {
+        if (mb & (1u << k)) {
+            const int i = d.identity ? r : __ldg(d.slot + r);
+            ++r;
+            const float y = to_float<TY>(static_cast<const TY*>(d.yrow)[i]);
+            const float qp = (KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, d.c.yoffg)) : y) * d.c.inv_zq;
+            w[k] = taylor_w(d.c, p[k], qp);
+        }
+    }
+}
+
+enum { kPickW = 0, kPickR = 1, kPickP = 2 };
+
+template <typename TZ, typename TY, int KIND>
+__device__ __forceinline__ void draw_x(const DrawCtx& d, int what, int jb, int seg_end, float (&p)[kVec], float (&w)[kVec], float (&x)[kVec]) {
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) { p[k] = 0.f; w[k] = 0.f; x[k] = 0.f; }
+    if (jb >= seg_end) return;
+    draw_pw<TZ, TY, KIND>(d, jb, p, w);
+#pragma unroll
+    for (int k = 0; k < kVec; ++k)
+        x[k] = what == kPickW ? w[k] : (what == kPickR ? fmaxf(0.f, p[k] - w[k] * d.c.inv_s) : p[k]);
+}
+
+template <typename TZ, typename TY, int KIND>
+__global__ void __launch_bounds__(kDT)
+rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
+    __shared__ double cdfW[kMaxSeg], cdfR[kMaxSeg], cdfP[kMaxSeg];
+    __shared__ float sums[2][kMaxChunks];
+    __shared__ float alpha_s;
+    __shared__ int res_tok[2];
+    __shared__ float res_p[2], res_w[2];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row = blockIdx.x / P.trials, t = blockIdx.x % P.trials;
+    if (!index_matches(P)) return;                 // kernel 1 has reported it
+    const float* rec = P.rec + (long long)row * kRecFloats;
+    const int nseg = C * kCW, Lw = Ls / kCW;
+
+    if (warp == 0) {   // prefix sums over the segments, fp64
+        double iw[2], ir[2], ip[2];
         float alpha_l = 0.f;
 #pragma unroll
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
-            sw[it] = sr[it] = sp[it] = 0.0;
+            iw[it] = ir[it] = ip[it] = 0.0;
             if (s < nseg) {
-                const Pub2* rp = cluster.map_shared_rank(&pub2, s / kCW);
-                const float oov = c.theta * segA[s];
-                const float w_s = oov + rp->Kw[s % kCW];
-                const float a_s = oov * c.inv_s + rp->ak[s % kCW];
-                sw[it] = (double)w_s;
-                sr[it] = (double)fmaxf(0.f, segP[s] - a_s);
-                sp[it] = (double)segP[s];
-                alpha_l += a_s;
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(rec + 16) + s);
+                iw[it] = (double)v.x; alpha_l += v.y; ir[it] = (double)v.z; ip[it] = (double)v.w;
             }
-        }
-        // inclusive scan over segments: lanes hold s = lane (it 0) and s = lane + 32 (it 1)
-        double iw[2], ir[2], ip[2];
-#pragma unroll
-        for (int it = 0; it < 2; ++it) {
-            iw[it] = sw[it]; ir[it] = sr[it]; ip[it] = sp[it];
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const double a = __shfl_up_sync(0xffffffffu, iw[it], o);
                 const double b = __shfl_up_sync(0xffffffffu, ir[it], o);
-                const double d = __shfl_up_sync(0xffffffffu, ip[it], o);
-                if (lane >= o) { iw[it] += a; ir[it] += b; ip[it] += d; }
+                const double e = __shfl_up_sync(0xffffffffu, ip[it], o);
+                if (lane >= o) { iw[it] += a; ir[it] += b; ip[it] += e; }
             }
         }
-        const double t0w = __shfl_sync(0xffffffffu, iw[0], 31), t0r = __shfl_sync(0xffffffffu, ir[0], 31),
-                     t0p = __shfl_sync(0xffffffffu, ip[0], 31);
-        iw[1] += t0w; ir[1] += t0r; ip[1] += t0p;
+        iw[1] += __shfl_sync(0xffffffffu, iw[0], 31);
+        ir[1] += __shfl_sync(0xffffffffu, ir[0], 31);
+        ip[1] += __shfl_sync(0xffffffffu, ip[0], 31);
 #pragma unroll
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
             if (s < nseg) { cdfW[s] = iw[it]; cdfR[s] = ir[it]; cdfP[s] = ip[it]; }
         }
         alpha_l = warp_sum(alpha_l);
-        if (lane == 0) bc[10] = alpha_l;
+        if (lane == 0) alpha_s = alpha_l;
     }
     __syncthreads();
     const double S_d = cdfW[nseg - 1], R_d = cdfR[nseg - 1], Pt_d = cdfP[nseg - 1];
-    if (crank == 0 && tid == 0) {
-        if (P.alpha) P.alpha[row] = bc[10];
-        if (P.theta) P.theta[row] = c.theta;
+    DrawCtx d;
+    d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
+    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
+    d.c.inv_s = __ldcg(rec + kRecInvS);
+    if (t == 0 && tid == 0) {
+        if (P.alpha) P.alpha[row] = alpha_s;
+        if (P.theta) P.theta[row] = d.c.theta;
         if (P.S) P.S[row] = (float)S_d;
         if (P.residual_mass) P.residual_mass[row] = (float)R_d;
     }
+    const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
+    d.zrow = zrow; d.yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
+    d.zvec = (reinterpret_cast<uintptr_t>(zrow) & 15u) == 0;
+    d.mask = P.mask; d.rank = P.rank; d.slot = P.slot; d.N = P.N; d.identity = P.header[kHdrIdentity] != 0;
 
-    // ---- draws: one trial per warp, kTrialBatch trials between exchanges ---------------------------
-    for (int t0 = 0; t0 < P.trials; t0 += kTrialBatch) {
-        const int t = t0 + warp;
-        const bool live = t < P.trials;
-        float u0 = 0.f, u1 = 0.f, u2 = 0.f;
-        int seg = 0;
-        if (live) {
-            const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
-            u0 = __ldg(u); u1 = __ldg(u + 1); u2 = __ldg(u + 2);
-            const double thr = (double)u0 * S_d;
-            seg = min(first_above(cdfW, nseg, thr), nseg - 1);
-            if (seg / kCW == crank) {
-                const float rem = (float)(thr - (seg ? cdfW[seg - 1] : 0.0));
-                const int a = (seg % kCW) * Lw;
-                float pd, wd;
-                int jl = pick_in_range<TZ, TY, KIND, kPickW>(c, a, a + Lw, rem, lane, pd, wd);
-                if (lane == 0) { pub3.d[warp] = jl < 0 ? j0 + a : j0 + jl; pub3.pd[warp] = pd; pub3.wd[warp] = wd; }
-            }
-        }
-        cluster.sync();                                                        // exchange 3: draft results
-        if (live) {
-            const Pub3* rp = cluster.map_shared_rank(&pub3, seg / kCW);
-            const int d = rp->d[warp];
-            const float pd = rp->pd[warp], wd = rp->wd[warp];
-            const float qd = wd * c.inv_s;
-            const float a_prob = (pd >= qd) ? 1.f : pd / qd;
-            const bool acc = u1 * qd < pd;
-            const long long o = (long long)row * P.trials + t;
-            if (seg / kCW == crank && lane == 0) {
-                if (P.draft_token) P.draft_token[o] = d;
-                if (P.accepted) P.accepted[o] = acc ? 1 : 0;
-                if (P.accept_prob) P.accept_prob[o] = a_prob;
-                if (acc && P.out_token) P.out_token[o] = d;
-            }
-            if (!acc) {
-                // residual draw from max(0, p - q~); if that has no mass, from p itself
-                const bool from_p = !(R_d > 0.0);
-                const double* cdf = from_p ? cdfP : cdfR;
-                const double thr = (double)u2 * (from_p ? Pt_d : R_d);
-                const int sr = min(first_above(cdf, nseg, thr), nseg - 1);
-                if (sr / kCW == crank) {
-                    const float rem = (float)(thr - (sr ? cdf[sr - 1] : 0.0));
-                    const int a = (sr % kCW) * Lw;
-                    float pp, ww;
-                    const int jl = from_p ? pick_in_range<TZ, TY, KIND, kPickP>(c, a, a + Lw, rem, lane, pp, ww)
-                                          : pick_in_range<TZ, TY, KIND, kPickR>(c, a, a + Lw, rem, lane, pp, ww);
-                    if (lane == 0 && P.out_token) P.out_token[o] = jl < 0 ? j0 + a : j0 + jl;
-                }
-            }
-        }
-        cluster.sync();                                                        // all remote reads of this batch done
+    const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
+    const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
+
+    // group 0 (warps 0-7): the draft draw from w; group 1 (warps 8-15): the residual draw, computed
+    // alongside (it is only used if the draft is rejected)
+    const int g = warp / kCW, wg = warp % kCW;
+    const bool from_p = !(R_d > 0.0);                 // p and q~ coincide: the replacement comes from p itself
+    const double* cdf = g == 0 ? cdfW : (from_p ? cdfP : cdfR);
+    const int what = g == 0 ? kPickW : (from_p ? kPickP : kPickR);
+    const double thr = g == 0 ? (double)u0 * S_d : (double)u2 * (from_p ? Pt_d : R_d);
+    const int seg = min(first_above(cdf, nseg, thr), nseg - 1);
+    const float rem = (float)(thr - (seg ? cdf[seg - 1] : 0.0));
+    const int seg_lo = (seg / kCW) * Ls + (seg % kCW) * Lw;
+    const int seg_end = min(P.N, seg_lo + Lw);
+    const int nch = (Lw + kSeg - 1) / kSeg;
+    for (int ch = wg; ch < nch; ch += kCW) {
+        float p[kVec], w[kVec], x[kVec];
+        draw_x<TZ, TY, KIND>(d, what, seg_lo + ch * kSeg + lane * kVec, seg_end, p, w, x);
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < kVec; ++k) s += x[k];
+        s = warp_sum(s);
+        if (lane == 0) sums[g][ch] = s;
     }
-    if (P.trials <= 0) cluster.sync();      // remote shared memory must outlive its readers
-    if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
+    __syncthreads();
+    {   // every warp finds the chunk of its group; the warp that owns it picks the token
+        float cum = 0.f, before = 0.f;
+        int chosen = -1, last_pos = -1;
+        for (int ch = 0; ch < nch; ++ch) {
+            const float s = sums[g][ch];
+            if (s > 0.f) {
+                if (chosen < 0 && cum + s > rem) { chosen = ch; before = cum; }
+                last_pos = ch;
+                cum += s;
+            }
+        }
+        float r_in = rem - before;
+        if (chosen < 0) { chosen = last_pos; r_in = INFINITY; }      // rounding: the last positive token
+        if (chosen < 0) {
+            if (wg == 0 && lane == 0) { res_tok[g] = seg_lo; res_p[g] = 0.f; res_w[g] = 0.f; }
+        } else if (chosen % kCW == wg) {
+            float p[kVec], w[kVec], x[kVec];
+            draw_x<TZ, TY, KIND>(d, what, seg_lo + chosen * kSeg + lane * kVec, seg_end, p, w, x);
+            int sel = pick_in_segment(x, r_in, lane);
+            if (sel < 0) sel = 0;
+            float ps = 0.f, ws = 0.f;
+#pragma unroll
+            for (int k = 0; k < kVec; ++k) if (k == (sel & (kVec - 1))) { ps = p[k]; ws = w[k]; }
+            ps = __shfl_sync(0xffffffffu, ps, sel / kVec);
+            ws = __shfl_sync(0xffffffffu, ws, sel / kVec);
+            if (lane == 0) { res_tok[g] = seg_lo + chosen * kSeg + sel; res_p[g] = ps; res_w[g] = ws; }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const int dtok = res_tok[0];
+        const float pd = res_p[0], qd = res_w[0] * d.c.inv_s;
+        const float a_prob = (pd >= qd) ? 1.f : pd / qd;
+        const bool acc = u1 * qd < pd;
+        const long long o = (long long)row * P.trials + t;
+        if (P.draft_token) P.draft_token[o] = dtok;
+        if (P.accepted) P.accepted[o] = acc ? 1 : 0;
+        if (P.accept_prob) P.accept_prob[o] = a_prob;
+        if (P.out_token) P.out_token[o] = acc ? dtok : res_tok[1];
+        if (P.accepted_len && P.accepted && P.counters) {
+            // the last position of a sequence to finish counts the accepted prefix (Algorithm 4 step 7)
+            const int b = row / P.positions;
+            __threadfence();
+            const int old = atomicAdd(P.counters + b * P.trials + t, 1);
+            if (old == P.positions - 1) {
+                __threadfence();
+                int k = 0;
+                const volatile uint8_t* af = P.accepted;
+                while (k < P.positions && af[((long long)b * P.positions + k) * P.trials + t]) ++k;
+                P.accepted_len[b * P.trials + t] = k;
+            }
+        }
+    }
 }
 
-template <typename TZ, typename TY, int KIND>
-static cudaError_t launch_one(const RowParams& P, int C, int Ls, int cap, size_t smem, cudaStream_t s) {
-    auto kern = rdk_cluster_kernel<TZ, TY, KIND>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)P.rows * C, 1, 1);
-    cfg.blockDim = dim3(kCT, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, P, C, Ls, cap);
-}
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+struct Geometry { int C, Ls, cap; size_t smem; };
 
-template <typename TZ, typename TY>
-static cudaError_t launch_kind_c(const RowParams& P, int kind, int C, int Ls, int cap, size_t smem, cudaStream_t s) {
-    return kind == RDK_LOGITS ? launch_one<TZ, TY, RDK_LOGITS>(P, C, Ls, cap, smem, s)
-                              : launch_one<TZ, TY, RDK_PROBS>(P, C, Ls, cap, smem, s);
-}
-
-cudaError_t launch_cluster_linear(const RowParams& P, int tz, int ty, int kind, cudaStream_t s) {
-    const size_t es = tz == RDK_F32 ? 4 : 2;
-    if (P.N < kMinClusterN || P.qtilde || P.rows <= 0) return cudaErrorNotSupported;
-    if ((reinterpret_cast<uintptr_t>(P.target) & 15u) || ((P.target_stride * (long long)es) & 15)) return cudaErrorNotSupported;
-    if ((long long)P.rows * kMaxC > 0x7fffffffLL) return cudaErrorNotSupported;
-    // cluster size: slices of at most 32 KB where eight CTAs allow it
+static bool plan_geometry(int N, int n, size_t es, Geometry& g) {
     int C = 1;
-    while (C < kMaxC && ((size_t)P.N * es + C - 1) / C > 32768) C *= 2;
-    const int per = (P.N + C - 1) / C;
+    while (C < kMaxC && ((size_t)N * es + C - 1) / C > 32768) C *= 2;      // slices of at most 32 KB if 8 CTAs allow
+    const int per = (N + C - 1) / C;
     const int Ls = (per + 255) / 256 * 256;
-    const long long expect = ((long long)P.n * Ls + P.N - 1) / P.N;
+    const long long expect = ((long long)n * Ls + N - 1) / N;
     long long cap = expect + expect / 8 + 64;
-    const long long most = P.n < Ls ? P.n : Ls;
+    const long long most = n < Ls ? n : Ls;
     if (cap > most) cap = most;
     cap = (cap + 31) / 32 * 32;
     const size_t zbytes = ((size_t)Ls * es + 127) & ~size_t(127);
     size_t smem = zbytes + (size_t)cap * sizeof(float2);
     if (smem > 200 * 1024) {
-        if (zbytes > 160 * 1024) return cudaErrorNotSupported;
+        if (zbytes > 160 * 1024) return false;
         cap = (long long)((200 * 1024 - zbytes) / sizeof(float2)) / 32 * 32;
         smem = zbytes + (size_t)cap * sizeof(float2);
     }
+    if ((Ls / kCW + kSeg - 1) / kSeg > kMaxChunks) return false;
+    g.C = C; g.Ls = Ls; g.cap = (int)cap; g.smem = smem;
+    return true;
+}
+
+template <typename TZ, typename TY, int KIND>
+static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_t s) {
+    auto kern = rdk_stream_kernel<TZ, TY, KIND>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P.rows * g.C, 1, 1);
+    cfg.blockDim = dim3(kCT, 1, 1);
+    cfg.dynamicSmemBytes = g.smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = g.C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kern, P, g.C, g.Ls, g.cap);
+    if (e != cudaSuccess) return e;
+    rdk_draw_kernel<TZ, TY, KIND><<<(unsigned)(P.rows * P.trials), kDT, 0, s>>>(P, g.C, g.Ls);
+    return cudaGetLastError();
+}
+
+template <typename TZ, typename TY>
+static cudaError_t launch_kind_c(const RowParams& P, int kind, const Geometry& g, cudaStream_t s) {
+    return kind == RDK_LOGITS ? launch_one<TZ, TY, RDK_LOGITS>(P, g, s) : launch_one<TZ, TY, RDK_PROBS>(P, g, s);
+}
+
+size_t cluster_workspace_bytes(int rows, int batch, int trials) {
+    return idx_align((size_t)rows * kRecFloats * sizeof(float)) + idx_align((size_t)batch * trials * sizeof(int32_t));
+}
+
+cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s) {
+    const size_t es = tz == RDK_F32 ? 4 : 2;
+    if (P.N < kMinClusterN || P.qtilde || P.rows <= 0 || P.trials <= 0 || !ws) return cudaErrorNotSupported;
+    if ((reinterpret_cast<uintptr_t>(P.target) & 15u) || ((P.target_stride * (long long)es) & 15)) return cudaErrorNotSupported;
+    if ((long long)P.rows * kMaxC > 0x7fffffffLL || (long long)P.rows * P.trials > 0x7fffffffLL) return cudaErrorNotSupported;
+    if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < cluster_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
+    Geometry g;
+    if (!plan_geometry(P.N, P.n, es, g)) return cudaErrorNotSupported;
+    P.rec = static_cast<float*>(ws);
+    P.counters = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + idx_align((size_t)P.rows * kRecFloats * sizeof(float)));
     if (tz == RDK_F32) {
-        if (ty == RDK_F32) return launch_kind_c<float, float>(P, kind, C, Ls, (int)cap, smem, s);
-        return launch_kind_c<float, __nv_bfloat16>(P, kind, C, Ls, (int)cap, smem, s);
+        if (ty == RDK_F32) return launch_kind_c<float, float>(P, kind, g, s);
+        return launch_kind_c<float, __nv_bfloat16>(P, kind, g, s);
     }
-    if (ty == RDK_F32) return launch_kind_c<__nv_bfloat16, float>(P, kind, C, Ls, (int)cap, smem, s);
-    return launch_kind_c<__nv_bfloat16, __nv_bfloat16>(P, kind, C, Ls, (int)cap, smem, s);
+    if (ty == RDK_F32) return launch_kind_c<__nv_bfloat16, float>(P, kind, g, s);
+    return launch_kind_c<__nv_bfloat16, __nv_bfloat16>(P, kind, g, s);
 }
 
 }  // namespace rdk

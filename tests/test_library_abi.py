@@ -53,20 +53,23 @@ def test_argument_errors_are_reported_on_the_host(B):
     pb.N, pb.n, pb.batch, pb.positions = 0, 4, 1, 1
     out = B.rdk_outputs()
     dummy = C.c_void_p(256)
-    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None)
+    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_INVALID_ARG and b"positive" in L.rdk_last_error()
     pb.N = 16
-    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None)
+    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_INVALID_ARG          # kept_index is NULL
     pb.kept_index = 256
-    st = L.rdk_sample_and_verify(C.byref(pb), 5, dummy, dummy, None, 0, dummy, 1, C.byref(out), None)
+    st = L.rdk_sample_and_verify(C.byref(pb), 5, dummy, dummy, None, 0, dummy, 1, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_INVALID_ARG          # unknown mode
-    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 0, C.byref(out), None)
+    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 0, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_INVALID_ARG          # trials < 1
-    st = L.rdk_sample_and_verify(C.byref(pb), 1, dummy, None, None, 0, dummy, 1, C.byref(out), None)
+    st = L.rdk_sample_and_verify(C.byref(pb), 1, dummy, None, None, 0, dummy, 1, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_INVALID_ARG          # precomputed mode without w
+    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None, 0, None)
+    assert st == B.RDK_ERR_WORKSPACE_TOO_SMALL  # the linear mode needs its workspace
+    assert L.rdk_sample_workspace_bytes(C.byref(pb), 0, 1) >= 1088 and L.rdk_sample_workspace_bytes(C.byref(pb), 1, 1) == 0
     pb.target_dtype = 9
-    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None)
+    st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_INVALID_ARG
     pb.target_dtype = 0
     pb.N = (1 << 21) + 1
