@@ -206,7 +206,7 @@ int rdk_redistribute_linear(const rdk_problem* problem, const void* target, cons
  *   out        see rdk_outputs
  *   ws         device workspace of rdk_sample_workspace_bytes(problem, mode, trials) bytes, 256-byte
  *              aligned (may be NULL when that size is 0).  It holds, between the two kernels of
- *              the linear path, one record of 1088 bytes per row (row scalars and per-segment sums
+ *              the linear path, one record of 2112 bytes per row (row scalars and per-segment sums
  *              of w, min(p, q~), max(0, p - q~), p) and one counter per (sequence, trial).
  * Arithmetic of the linear mode: fp32; for N >= 4096 the quotient 1 / (N + p_j) is expanded as
  * (1/N)(1 - x + x^2), x = p_j / N <= 2^-12 (relative truncation below 2^-36), otherwise divided.

@@ -25,7 +25,7 @@ struct RowParams {
     int32_t* counters;     // per (sequence, trial) arrival counters in the workspace
 };
 
-constexpr int kRecFloats = 16 + 4 * 64;   // per-row record: 16 scalars + 4 sums for each of up to 64 segments
+constexpr int kRecFloats = 16 + 4 * 128;  // per-row record: 16 scalars + 4 sums for each of up to 128 segments
 
 // running (max, sum) pair of a soft-max denominator; `b` is a second sum on the same scale
 struct MS { float m, s, b; };

@@ -1,8 +1,9 @@
 // Two-kernel form of the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8) for N >= 4096.
 //
-// Kernel 1 (rdk_stream_kernel): one thread-block cluster of C CTAs per row.  CTA c brings its slice
-// of the target logits into shared memory with TMA bulk copies, so the row is read from HBM exactly
-// once; the C partial results are exchanged once through distributed shared memory.  It leaves a
+// Kernel 1 (rdk_stream_kernel): persistent thread-block clusters of C CTAs, one row at a time.
+// CTA c brings its slice of the target logits (and the matching drafter values) into shared memory
+// with TMA bulk copies, so a row is read from HBM exactly once; the C partial results are exchanged
+// once per row through distributed shared memory, while the next row's copies are in flight.  It leaves a
 // small record per row in the workspace: the row's scalars and, for each of the C*8 contiguous
 // token segments, the sums of w, of min(p, q~), of max(0, p - q~) and of p.
 // Kernel 2 (rdk_draw_kernel): one CTA per (row, trial) turns the record into draws: it locates the
@@ -33,15 +34,16 @@ constexpr int kMaxC = 8;             // portable cluster size
 constexpr int kMaxSeg = kMaxC * kCW;
 constexpr int kMinClusterN = 4096;
 constexpr unsigned kSpinLimit = 1u << 22;
-constexpr int kDT = 512;             // threads per CTA of kernel 2: 8 warps for the draft, 8 for the residual
+constexpr int kDT = 256;             // threads per CTA of kernel 2: 4 warps for the draft, 4 for the residual
+constexpr int kGW = kDT / 64;        // warps per group of kernel 2
 constexpr int kMaxChunks = 128;      // 256-token chunks per segment (N <= 2^21)
 
 // record layout (floats): 16 scalars, then 4 per segment
 enum { kRecOffg = 0, kRecInvZp, kRecYoffg, kRecInvZq, kRecTheta, kRecInvN, kRecInvS, kRecS };
 
-struct Pub1 {    // per-CTA partials, published before the exchange
+struct Pub1 {    // one CTA's partials; every CTA holds a copy of all C of them after the exchange
     float m, my;
-    float E1[kCW], E2[kCW], K1[kCW], K2[kCW], Zq[kCW], th[kCW], q2[kCW];
+    float E1[kCW], E2[kCW], K1[kCW], K2[kCW], Zq[kCW], th[kCW];
 };
 
 struct Scal { float offg, inv_zp, yoffg, inv_zq, theta, inv_n, inv_s; };
@@ -82,27 +84,139 @@ __device__ __forceinline__ bool index_matches(const RowParams& P) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// kernel 1
+// kernel 1: persistent clusters.  Cluster g takes rows g, g + G, g + 2G, ...; while a row's
+// partial results are exchanged and its kept tokens are revisited, the bulk copies of the next
+// row's slice are already in flight.
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(*reinterpret_cast<unsigned long long*>(&d))
+        : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)),
+          "l"(*reinterpret_cast<unsigned long long*>(&c)));
+    return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    float2 d;
+    asm("add.rn.f32x2 %0, %1, %2;"
+        : "=l"(*reinterpret_cast<unsigned long long*>(&d))
+        : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+    return d;
+}
+
+// running maximum over 8 consecutive logits in shared memory
+template <typename TZ> struct MaxAcc;
+template <> struct MaxAcc<float> {
+    float m = -INFINITY;
+    __device__ __forceinline__ void push(const float* zb, int jl) {
+        const float4 a = *reinterpret_cast<const float4*>(zb + jl);
+        const float4 b = *reinterpret_cast<const float4*>(zb + jl + 4);
+        m = fmaxf(fmaxf(fmaxf(m, a.x), fmaxf(a.y, a.z)), fmaxf(fmaxf(a.w, b.x), fmaxf(b.y, fmaxf(b.z, b.w))));
+    }
+    __device__ __forceinline__ float result() const { return m; }
+};
+template <> struct MaxAcc<__nv_bfloat16> {
+    __nv_bfloat162 m2 = __float2bfloat162_rn(-INFINITY);
+    __device__ __forceinline__ void push(const __nv_bfloat16* zb, int jl) {
+        const uint4 q = *reinterpret_cast<const uint4*>(zb + jl);
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.z));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+    }
+    __device__ __forceinline__ float result() const { return fmaxf(__low2float(m2), __high2float(m2)); }
+};
+
+// sum of e = 2^(z log2e + off) and of e^2 over 8 consecutive logits in shared memory (packed fp32 pairs)
+template <typename TZ>
+__device__ __forceinline__ void exp_sums8(const TZ* zb, int jl, float2 scale, float2 off, float2& E1, float2& E2);
+template <>
+__device__ __forceinline__ void exp_sums8<__nv_bfloat16>(const __nv_bfloat16* zb, int jl, float2 scale, float2 off, float2& E1, float2& E2) {
+    const uint4 q = *reinterpret_cast<const uint4*>(zb + jl);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 x = ffma2(make_float2(bf16_lo(w[k]), bf16_hi(w[k])), scale, off);
+        const float2 e = make_float2(ex2(x.x), ex2(x.y));
+        E1 = fadd2(E1, e);
+        E2 = ffma2(e, e, E2);
+    }
+}
+template <>
+__device__ __forceinline__ void exp_sums8<float>(const float* zb, int jl, float2 scale, float2 off, float2& E1, float2& E2) {
+    const float4 a = *reinterpret_cast<const float4*>(zb + jl);
+    const float4 b = *reinterpret_cast<const float4*>(zb + jl + 4);
+    const float2 v[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y), make_float2(b.z, b.w)};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 x = ffma2(v[k], scale, off);
+        const float2 e = make_float2(ex2(x.x), ex2(x.y));
+        E1 = fadd2(E1, e);
+        E2 = ffma2(e, e, E2);
+    }
+}
+
+__device__ __forceinline__ void mbar_wait(unsigned long long* bar, uint32_t parity, int* fail) {
+    unsigned spins = 0;
+    uint32_t done = 0;
+    while (!done) {
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (!done && ++spins > kSpinLimit) { atomicExch(fail, 1); break; }   // give up: the host reads RDK_ERR_TIMEOUT
+    }
+}
+
+// One thread: arm `bar` for `bytes` and issue the bulk copies (bytes is a multiple of 16, may be 0).
+__device__ __forceinline__ void bulk_load(unsigned long long* bar, void* dst, const void* src, uint32_t bytes) {
+    if (bytes == 0) {
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+        return;
+    }
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+    for (uint32_t off = 0; off < bytes; off += 16384u) {
+        const uint32_t sz = min(16384u, bytes - off);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_u32(static_cast<char*>(dst) + off)), "l"(static_cast<const char*>(src) + off), "r"(sz),
+                       "r"(smem_u32(bar)) : "memory");
+    }
+}
+
+// How the first `kcs` drafter values of a row's rank range are laid out in a y buffer: element il
+// sits at index sh + il, so that the 16-byte aligned middle part can be bulk-copied.
+struct YPlan { int sh, head, mid, tail; };
+template <typename TY>
+__device__ __forceinline__ YPlan plan_y(const TY* src, int kcs) {
+    YPlan p;
+    const uint32_t a = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 15u);
+    p.sh = (int)(a / sizeof(TY));
+    p.head = min(kcs, (int)(((16u - a) & 15u) / sizeof(TY)));
+    const int rest = kcs - p.head;
+    p.mid = (int)(((size_t)rest * sizeof(TY) & ~size_t(15)) / sizeof(TY));
+    p.tail = rest - p.mid;
+    return p;
+}
+
 template <typename TZ, typename TY, int KIND>
-__global__ void __launch_bounds__(kCT)
-rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap) {
+__global__ void __launch_bounds__(kCT, 2)
+rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, const int G) {
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(128) unsigned char dsm[];
+    const size_t zb_bytes = ((size_t)Ls * sizeof(TZ) + 127) & ~size_t(127);
+    const size_t yb_bytes = ((size_t)(cap + 16) * sizeof(TY) + 127) & ~size_t(127);
     TZ* zbuf = reinterpret_cast<TZ*>(dsm);
-    float2* cache = reinterpret_cast<float2*>(dsm + (((size_t)Ls * sizeof(TZ) + 127) & ~size_t(127)));
+    TY* ybuf[2] = {reinterpret_cast<TY*>(dsm + zb_bytes), reinterpret_cast<TY*>(dsm + zb_bytes + yb_bytes)};
+    int32_t* idsb = reinterpret_cast<int32_t*>(dsm + zb_bytes + 2 * yb_bytes);
+    float* ezb = reinterpret_cast<float*>(idsb + cap);
 
-    __shared__ Pub1 pub1;
-    __shared__ float segA[kCW], segP[kCW];
-    __shared__ float bc[12];
+    __shared__ Pub1 all1[2][kMaxC];        // [row parity][source CTA], written by the source CTAs
     __shared__ float redm[kCW], redy[kCW];
     __shared__ int rk[kCW + 1];
-    __shared__ __align__(8) unsigned long long bar;
+    __shared__ __align__(8) unsigned long long zbar, ybar[2];
     __shared__ int fail;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int crank = (int)cluster.block_rank();
-    const int row = blockIdx.x / C;
+    const int cid = blockIdx.x / C;
 
     if (!index_matches(P)) {   // same decision in every CTA of the grid; nothing is in flight yet
         if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
@@ -114,213 +228,219 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap) {
     const int j0 = crank * Ls;
     const int len = max(0, min(P.N - j0, Ls));
     const int Lw = Ls / kCW;
-    const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
-    const TY* yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
-
-    // ---- stage the slice: one thread issues the bulk copies, everybody pads the tail ------------
     const int len8 = len & ~(kVec - 1);
-    const uint32_t bytes = (uint32_t)len8 * (uint32_t)sizeof(TZ);
+    const uint32_t zbytes = (uint32_t)len8 * (uint32_t)sizeof(TZ);
+
     if (tid == 0) {
         fail = 0;
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&zbar)));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&ybar[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&ybar[1])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (bytes) {
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&bar)), "r"(bytes) : "memory");
-            const char* src = reinterpret_cast<const char*>(zrow + j0);
-            for (uint32_t off = 0; off < bytes; off += 16384u) {
-                const uint32_t sz = min(16384u, bytes - off);
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(smem_u32(dsm + off)), "l"(src + off), "r"(sz), "r"(smem_u32(&bar)) : "memory");
-            }
-        }
     }
     if (tid <= kCW) rk[tid] = rank_at(P, min(P.N, j0 + tid * Lw), n_valid);   // rank at the warp range borders
-    for (int idx = len8 + tid; idx < Ls; idx += kCT) zbuf[idx] = idx < len ? zrow[j0 + idx] : neg_inf<TZ>();
+    for (int idx = len + tid; idx < Ls; idx += kCT) zbuf[idx] = neg_inf<TZ>();   // beyond the vocabulary: weight 0
     __syncthreads();
-
-    // ---- drafter slice: (local token index, raw value) into the cache, running max ---------------
     const int r0 = rk[0];
-    const int kc = rk[kCW] - r0;
-    float my_t = -INFINITY;
-#pragma unroll 4
-    for (int il = tid; il < kc; il += kCT) {
-        const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
-        const float y = to_float<TY>(yrow[i]);
-        const int jl = __ldg(P.ids + i) - j0;
-        if (il < cap) cache[il] = make_float2(__int_as_float(jl), y);
-        if (KIND == RDK_LOGITS) my_t = fmaxf(my_t, y);
-    }
+    const int kc = rk[kCW] - r0;          // kept tokens of this slice
+    const int kcs = min(kc, cap);         // ... of which this many are staged in shared memory
 
-    if (bytes) {   // bounded wait for the bulk copies
-        unsigned spins = 0;
-        uint32_t done = 0;
-        while (!done) {
-            asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                         : "=r"(done) : "r"(smem_u32(&bar)), "r"(0u) : "memory");
-            if (!done && ++spins > kSpinLimit) { atomicExch(&fail, 1); break; }
+    // Loads of one row: z slice and the drafter values of the slice's rank range.
+    auto issue_loads = [&](int row, int b) {
+        const TZ* zsrc = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride + j0;
+        const TY* ysrc = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
+        if (tid < len - len8) zbuf[len8 + tid] = zsrc[len8 + tid];                 // ragged end of the slice
+        if (identity) {
+            const YPlan yp = plan_y<TY>(ysrc + r0, kcs);
+            if (tid == kCT - 32) {
+                bulk_load(&zbar, zbuf, zsrc, zbytes);
+                bulk_load(&ybar[b], ybuf[b] + yp.sh + yp.head, ysrc + r0 + yp.head, (uint32_t)(yp.mid * sizeof(TY)));
+            }
+            if (tid >= 32 && tid < 32 + yp.head) { const int il = tid - 32; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
+            if (tid >= 64 && tid < 64 + yp.tail) { const int il = yp.head + yp.mid + tid - 64; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
+        } else {
+            if (tid == kCT - 32) { bulk_load(&zbar, zbuf, zsrc, zbytes); bulk_load(&ybar[b], nullptr, nullptr, 0); }
+            for (int il = tid; il < kcs; il += kCT) ybuf[b][il] = ysrc[__ldg(P.slot + r0 + il)];
         }
-    }
+    };
+    auto y_shift = [&](int row) -> int {
+        if (!identity) return 0;
+        const TY* ysrc = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride + r0;
+        return (int)((reinterpret_cast<uintptr_t>(ysrc) & 15u) / sizeof(TY));
+    };
 
-    // ---- slice maximum of z -------------------------------------------------------------------
+    if (cid < P.rows) issue_loads(cid, 0);
+    // token ids of the slice's kept tokens, in rank order: the same for every row
+    for (int il = tid; il < kcs; il += kCT) idsb[il] = __ldg(P.ids + (identity ? r0 + il : __ldg(P.slot + r0 + il)));
+
     const int wa = warp * Lw, wb = wa + Lw;
-    float mz_t = -INFINITY;
-    for (int cs = wa; cs < wb; cs += kSeg) {
-        const int jl = cs + lane * kVec;
-        if (jl < wb) {
-            float z[kVec];
-            lds8<TZ>(zbuf, jl, z);
-#pragma unroll
-            for (int k = 0; k < kVec; ++k) mz_t = fmaxf(mz_t, z[k]);
-        }
-    }
-    mz_t = warp_max(mz_t);
-    my_t = warp_max(my_t);
-    if (lane == 0) { redm[warp] = mz_t; redy[warp] = my_t; }
-    __syncthreads();
-    float m_c = redm[0], my_c = redy[0];
-#pragma unroll
-    for (int k = 1; k < kCW; ++k) { m_c = fmaxf(m_c, redm[k]); my_c = fmaxf(my_c, redy[k]); }
-    if (KIND == RDK_PROBS) my_c = 0.f;
+    const int rw0 = rk[warp] - r0, rw1 = rk[warp + 1] - r0;
+    const int rw1s = min(rw1, kcs);       // staged part of the warp's kept tokens
+    const int nseg = C * kCW;
+    const float inv_n = 1.f / (float)P.N;
 
-    // ---- soft-max sweep: sum e and sum e^2 over the warp's token range --------------------------
-    const float zoff_c = -m_c * kLog2e, yoff_c = -my_c * kLog2e;
-    float E1 = 0.f, E2 = 0.f;
-    if (m_c > -INFINITY) {
+    int it = 0;
+    for (int row = cid; row < P.rows; row += G, ++it) {
+        const int b = it & 1;
+        const TY* yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
+        const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
+        const TY* yb = ybuf[b] + y_shift(row);
+        mbar_wait(&zbar, (uint32_t)(it & 1), &fail);
+        mbar_wait(&ybar[b], (uint32_t)((it >> 1) & 1), &fail);
+        __syncthreads();                  // the few elements staged with plain stores are visible
+
+        // ---- maxima of the slice's logits and of its drafter values ---------------------------------
+        MaxAcc<TZ> mz;
         for (int cs = wa; cs < wb; cs += kSeg) {
             const int jl = cs + lane * kVec;
-            if (jl < wb) {
-                float z[kVec];
-                lds8<TZ>(zbuf, jl, z);
+            if (jl < wb) mz.push(zbuf, jl);
+        }
+        float my_t = -INFINITY;
+        if (KIND == RDK_LOGITS) {
+            for (int il = tid; il < kcs; il += kCT) my_t = fmaxf(my_t, to_float<TY>(yb[il]));
+            for (int il = cap + tid; il < kc; il += kCT)
+                my_t = fmaxf(my_t, to_float<TY>(yrow[identity ? r0 + il : __ldg(P.slot + r0 + il)]));
+        }
+        const float mz_w = warp_max(mz.result());
+        my_t = warp_max(my_t);
+        if (lane == 0) { redm[warp] = mz_w; redy[warp] = my_t; }
+        __syncthreads();
+        float m_c = redm[0], my_c = redy[0];
 #pragma unroll
-                for (int k = 0; k < kVec; ++k) {
-                    const float e = ex2(fmaf(z[k], kLog2e, zoff_c));
-                    E1 += e;
-                    E2 = fmaf(e, e, E2);
+        for (int k = 1; k < kCW; ++k) { m_c = fmaxf(m_c, redm[k]); my_c = fmaxf(my_c, redy[k]); }
+        if (KIND == RDK_PROBS) my_c = 0.f;
+
+        // ---- soft-max sweep: sum e and sum e^2 over the warp's token range ----------------------------
+        const float zoff_c = -m_c * kLog2e, yoff_c = -my_c * kLog2e;
+        float E1 = 0.f, E2 = 0.f;
+        if (m_c > -INFINITY) {
+            float2 e1 = make_float2(0.f, 0.f), e2 = make_float2(0.f, 0.f);
+            const float2 sc = make_float2(kLog2e, kLog2e), of = make_float2(zoff_c, zoff_c);
+#pragma unroll 2
+            for (int cs = wa; cs < wb; cs += kSeg) {
+                const int jl = cs + lane * kVec;
+                if (jl < wb) exp_sums8<TZ>(zbuf, jl, sc, of, e1, e2);
+            }
+            E1 = e1.x + e1.y; E2 = e2.x + e2.y;
+        }
+        // ---- kept tokens of the warp's range: e_z (cached), e_y, their sums -----------------------------
+        float K1 = 0.f, K2 = 0.f, Zq = 0.f, th = 0.f;
+#pragma unroll 2
+        for (int il = rw0 + lane; il < rw1s; il += 32) {
+            const float ez = ex2(fmaf(to_float<TZ>(zbuf[idsb[il] - j0]), kLog2e, zoff_c));
+            const float y = to_float<TY>(yb[il]);
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            K1 += ez; K2 = fmaf(ez, ez, K2); Zq += ey; th = fmaf(ez, ey, th);
+            ezb[il] = ez;
+        }
+        for (int il = max(rw0, cap) + lane; il < rw1; il += 32) {      // kept tokens that did not fit the cache
+            const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
+            const float ez = ex2(fmaf(to_float<TZ>(zbuf[__ldg(P.ids + i) - j0]), kLog2e, zoff_c));
+            const float y = to_float<TY>(yrow[i]);
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            K1 += ez; K2 = fmaf(ez, ez, K2); Zq += ey; th = fmaf(ez, ey, th);
+        }
+        E1 = warp_sum(E1); E2 = warp_sum(E2); K1 = warp_sum(K1); K2 = warp_sum(K2);
+        Zq = warp_sum(Zq); th = warp_sum(th);
+        // push this warp's sums into every CTA of the cluster (lane c writes to CTA c)
+        if (lane < C) {
+            Pub1* rp = cluster.map_shared_rank(&all1[b][crank], lane);
+            rp->E1[warp] = E1; rp->E2[warp] = E2; rp->K1[warp] = K1; rp->K2[warp] = K2; rp->Zq[warp] = Zq; rp->th[warp] = th;
+            if (warp == 0) { rp->m = m_c; rp->my = my_c; }
+        }
+        __syncthreads();                  // every warp is done with zbuf: the next row may stream in
+        cluster.barrier_arrive();
+        if (row + G < P.rows) issue_loads(row + G, b ^ 1);
+        cluster.barrier_wait();                                                // the one exchange per row
+
+        // ---- combine the C partials: every warp does it for itself, in the same order everywhere ----
+        Scal c;
+        float fz, fy, segA_w = 0.f, segP_w = 0.f, S_row;
+        {
+            float mc = -INFINITY, myc = -INFINITY;
+            if (lane < C) { mc = all1[b][lane].m; myc = all1[b][lane].my; }
+            const float m = warp_max(mc), my = warp_max(myc);
+            const float f_l = mc > -INFINITY ? ex2((mc - m) * kLog2e) : 0.f;
+            const float g_l = myc > -INFINITY ? ex2((myc - my) * kLog2e) : 0.f;
+            float e1[kMaxSeg / 32], e2[kMaxSeg / 32], k1[kMaxSeg / 32], k2[kMaxSeg / 32];
+            float tZp = 0.f, tE2 = 0.f, tZq = 0.f, tTh = 0.f;
+#pragma unroll
+            for (int q = 0; q < kMaxSeg / 32; ++q) {
+                const int s = lane + 32 * q;
+                const bool valid = s < nseg;
+                const int cc = valid ? s / kCW : 0, w = s % kCW;
+                const float f = __shfl_sync(0xffffffffu, f_l, cc), g = __shfl_sync(0xffffffffu, g_l, cc);
+                e1[q] = e2[q] = k1[q] = k2[q] = 0.f;
+                if (valid) {
+                    const Pub1* rp = &all1[b][cc];
+                    e1[q] = f * rp->E1[w]; e2[q] = f * f * rp->E2[w];
+                    k1[q] = f * rp->K1[w]; k2[q] = f * f * rp->K2[w];
+                    tZp += e1[q]; tE2 += e2[q];
+                    tZq += g * rp->Zq[w]; tTh += f * g * rp->th[w];
                 }
             }
-        }
-    }
-    // ---- kept tokens of the warp's range: e_z, e_y, their sums ------------------------------------
-    const int rw0 = rk[warp] - r0, rw1 = rk[warp + 1] - r0;
-    float K1 = 0.f, K2 = 0.f, Zq = 0.f, th = 0.f, q2 = 0.f;
-#pragma unroll 2
-    for (int il = rw0 + lane; il < rw1; il += 32) {
-        int jl;
-        float y;
-        if (il < cap) { const float2 v = cache[il]; jl = __float_as_int(v.x); y = v.y; }
-        else {
-            const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
-            jl = __ldg(P.ids + i) - j0;
-            y = to_float<TY>(yrow[i]);
-        }
-        const float ez = ex2(fmaf(to_float<TZ>(zbuf[jl]), kLog2e, zoff_c));
-        const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
-        K1 += ez;
-        K2 = fmaf(ez, ez, K2);
-        Zq += ey;
-        th = fmaf(ez, ey, th);
-        q2 = fmaf(ez * ez, ey, q2);
-        if (il < cap) cache[il] = make_float2(ez, ey);
-    }
-    E1 = warp_sum(E1); E2 = warp_sum(E2); K1 = warp_sum(K1); K2 = warp_sum(K2);
-    Zq = warp_sum(Zq); th = warp_sum(th); q2 = warp_sum(q2);
-    if (lane == 0) {
-        pub1.E1[warp] = E1; pub1.E2[warp] = E2; pub1.K1[warp] = K1; pub1.K2[warp] = K2;
-        pub1.Zq[warp] = Zq; pub1.th[warp] = th; pub1.q2[warp] = q2;
-    }
-    if (tid == 0) { pub1.m = m_c; pub1.my = my_c; }
-    cluster.sync();                                                            // the one exchange
-
-    // ---- combine the C partials (warp 0 of every CTA, same order everywhere) ----------------------
-    const int nseg = C * kCW;
-    if (warp == 0) {
-        float mc = -INFINITY, myc = -INFINITY;
-        if (lane < C) {
-            const Pub1* rp = cluster.map_shared_rank(&pub1, lane);
-            mc = rp->m; myc = rp->my;
-        }
-        const float m = warp_max(mc), my = warp_max(myc);
-        const float f_l = mc > -INFINITY ? ex2((mc - m) * kLog2e) : 0.f;
-        const float g_l = myc > -INFINITY ? ex2((myc - my) * kLog2e) : 0.f;
-        float e1[2], e2[2], k1[2], k2[2];
-        float tZp = 0.f, tE2 = 0.f, tZq = 0.f, tTh = 0.f, tQ2 = 0.f;
+            tZp = warp_sum(tZp); tE2 = warp_sum(tE2); tZq = warp_sum(tZq); tTh = warp_sum(tTh);
+            const float inv_zp = 1.f / tZp, inv_zq = 1.f / tZq;
+            const float theta = tTh * inv_zp * inv_zq;
+            const float P2 = tE2 * inv_zp * inv_zp;
+            S_row = fmaf(-theta * P2 * inv_n, inv_n, 1.f);           // 1 - theta sum p^2 / N^2 (next term below 1/N^2)
+            // this warp's own segment: total p mass, and sum over its not-kept tokens of p / (N + p)
+            const int s_me = crank * kCW + warp;
 #pragma unroll
-        for (int it = 0; it < 2; ++it) {
-            const int s = lane + 32 * it;
-            const bool valid = s < nseg;
-            const int c = valid ? s / kCW : 0, w = s % kCW;
-            const float f = __shfl_sync(0xffffffffu, f_l, c), g = __shfl_sync(0xffffffffu, g_l, c);
-            e1[it] = e2[it] = k1[it] = k2[it] = 0.f;
-            if (valid) {
-                const Pub1* rp = cluster.map_shared_rank(&pub1, c);
-                e1[it] = f * rp->E1[w]; e2[it] = f * f * rp->E2[w];
-                k1[it] = f * rp->K1[w]; k2[it] = f * f * rp->K2[w];
-                tZp += e1[it]; tE2 += e2[it];
-                tZq += g * rp->Zq[w]; tTh += f * g * rp->th[w]; tQ2 += f * f * g * rp->q2[w];
+            for (int q = 0; q < kMaxSeg / 32; ++q) {
+                const float Po = fmaxf(0.f, e1[q] - k1[q]) * inv_zp;
+                const float P2o = fmaxf(0.f, e2[q] - k2[q]) * inv_zp * inv_zp;
+                const float pa = e1[q] * inv_zp, aa = inv_n * (Po - inv_n * P2o);
+                const float pb_ = __shfl_sync(0xffffffffu, pa, s_me & 31), ab_ = __shfl_sync(0xffffffffu, aa, s_me & 31);
+                if ((s_me >> 5) == q) { segP_w = pb_; segA_w = ab_; }
             }
+            const float f_me = __shfl_sync(0xffffffffu, f_l, crank), g_me = __shfl_sync(0xffffffffu, g_l, crank);
+            c.offg = -m * kLog2e; c.inv_zp = inv_zp; c.yoffg = -my * kLog2e; c.inv_zq = inv_zq; c.theta = theta;
+            c.inv_n = inv_n; c.inv_s = 1.f / S_row;
+            fz = f_me * inv_zp; fy = (KIND == RDK_LOGITS ? g_me : 1.f) * inv_zq;
         }
-        tZp = warp_sum(tZp); tE2 = warp_sum(tE2); tZq = warp_sum(tZq); tTh = warp_sum(tTh); tQ2 = warp_sum(tQ2);
-        const float inv_zp = 1.f / tZp, inv_zq = 1.f / tZq, inv_n = 1.f / (float)P.N;
-        const float theta = tTh * inv_zp * inv_zq;
-        const float P2 = tE2 * inv_zp * inv_zp, Q2 = tQ2 * inv_zp * inv_zp * inv_zq;
-        const float S = fmaf((Q2 - theta * P2) * inv_n, inv_n, 1.f);
-#pragma unroll
-        for (int it = 0; it < 2; ++it) {
-            const int s = lane + 32 * it;
-            if (s < nseg && s / kCW == crank) {
-                const float Po = fmaxf(0.f, e1[it] - k1[it]) * inv_zp;
-                const float P2o = fmaxf(0.f, e2[it] - k2[it]) * inv_zp * inv_zp;
-                segP[s % kCW] = e1[it] * inv_zp;
-                segA[s % kCW] = inv_n * (Po - inv_n * P2o);       // sum over not-kept tokens of p / (N + p)
-            }
-        }
-        const float f_me = __shfl_sync(0xffffffffu, f_l, crank), g_me = __shfl_sync(0xffffffffu, g_l, crank);
-        if (lane == 0) {
-            bc[0] = -m * kLog2e; bc[1] = inv_zp; bc[2] = -my * kLog2e; bc[3] = inv_zq; bc[4] = theta;
-            bc[5] = inv_n; bc[6] = 1.f / S; bc[7] = f_me * inv_zp; bc[8] = (KIND == RDK_LOGITS ? g_me : 1.f) * inv_zq;
-            bc[9] = S;
-        }
-    }
-    cluster.barrier_arrive();          // this thread reads no remote shared memory from here on
-    __syncthreads();
-    Scal c;
-    c.offg = bc[0]; c.inv_zp = bc[1]; c.yoffg = bc[2]; c.inv_zq = bc[3]; c.theta = bc[4]; c.inv_n = bc[5]; c.inv_s = bc[6];
-    const float fz = bc[7], fy = bc[8];
 
-    // ---- kept tokens again: p, w, min(p, q~) ---------------------------------------------------
-    float Kw = 0.f, ak = 0.f;
+        // ---- kept tokens again: sum of min(p, q~) --------------------------------------------------
+        float ak = 0.f;
 #pragma unroll 2
-    for (int il = rw0 + lane; il < rw1; il += 32) {
-        float ez, ey;
-        if (il < cap) { const float2 v = cache[il]; ez = v.x; ey = v.y; }
-        else {
+        for (int il = rw0 + lane; il < rw1s; il += 32) {
+            const float y = to_float<TY>(yb[il]);
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            const float p = ezb[il] * fz;
+            ak += fminf(p, taylor_w(c, p, ey * fy) * c.inv_s);
+        }
+        for (int il = max(rw0, cap) + lane; il < rw1; il += 32) {
             const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
-            ez = ex2(fmaf(to_float<TZ>(zbuf[__ldg(P.ids + i) - j0]), kLog2e, zoff_c));
+            const float ez = ex2(fmaf(to_float<TZ>(zrow[__ldg(P.ids + i)]), kLog2e, zoff_c));
             const float y = to_float<TY>(yrow[i]);
-            ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            const float p = ez * fz;
+            ak += fminf(p, taylor_w(c, p, ey * fy) * c.inv_s);
         }
-        const float p = ez * fz, qp = ey * fy;
-        const float w = taylor_w(c, p, qp);
-        Kw += w;
-        ak += fminf(p, w * c.inv_s);
-    }
-    Kw = warp_sum(Kw); ak = warp_sum(ak);
+        ak = warp_sum(ak);
 
-    // ---- the row's record ---------------------------------------------------------------------
-    float* rec = P.rec + (long long)row * kRecFloats;
-    if (lane == 0) {
-        const float oov = c.theta * segA[warp];
-        const float w_s = oov + Kw;
-        const float a_s = oov * c.inv_s + ak;
-        reinterpret_cast<float4*>(rec + 16)[crank * kCW + warp] = make_float4(w_s, a_s, fmaxf(0.f, segP[warp] - a_s), segP[warp]);
-    }
-    if (crank == 0) {
-        if (tid < 8) rec[tid] = tid < 7 ? bc[tid] : bc[9];
-        if (P.counters && row % P.positions == 0)
-            for (int t = tid; t < P.trials; t += kCT) P.counters[(row / P.positions) * P.trials + t] = 0;
+        // ---- the row's record -------------------------------------------------------------------------
+        float* rec = P.rec + (long long)row * kRecFloats;
+        if (lane == 0) {
+            // sum over the segment's kept tokens of w = (q' + theta x)(1 - x + x^2), x = p / N, from the
+            // moments of pass 1 (terms of relative size x^2 <= 2^-24 dropped)
+            const float xs = fz * c.inv_n;
+            const float Kw = fy * Zq - fy * xs * th + c.theta * (xs * K1 - xs * xs * K2);
+            const float oov = c.theta * segA_w;
+            const float a_s = oov * c.inv_s + ak;
+            reinterpret_cast<float4*>(rec + 16)[crank * kCW + warp] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP_w - a_s), segP_w);
+        }
+        if (crank == 0) {
+            if (tid == 0) {
+                rec[kRecOffg] = c.offg; rec[kRecInvZp] = c.inv_zp; rec[kRecYoffg] = c.yoffg; rec[kRecInvZq] = c.inv_zq;
+                rec[kRecTheta] = c.theta; rec[kRecInvN] = c.inv_n; rec[kRecInvS] = c.inv_s; rec[kRecS] = S_row;
+            }
+            if (P.counters && row % P.positions == 0)
+                for (int t = tid; t < P.trials; t += kCT) P.counters[(row / P.positions) * P.trials + t] = 0;
+        }
     }
     if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
-    cluster.barrier_wait();            // remote shared memory must outlive its readers
+    cluster.sync();                        // remote shared memory must outlive its readers
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -339,6 +459,7 @@ __device__ __forceinline__ void draw_pw(const DrawCtx& d, int jb, float (&p)[kVe
     float z[kVec];
     load8<TZ>(static_cast<const TZ*>(d.zrow), jb, d.N, d.zvec, -INFINITY, z);
     const uint32_t word = __ldg(d.mask + (jb >> 5));
+    const int rbase = __ldg(d.rank + (jb >> 5));          // issued together with the mask and the logits
     const int sh = jb & 31;
     const uint32_t mb = (word >> sh) & 0xffu;
 #pragma unroll
@@ -347,7 +468,7 @@ __device__ __forceinline__ void draw_pw(const DrawCtx& d, int jb, float (&p)[kVe
         w[k] = taylor_w(d.c, p[k], 0.f);
     }
     if (!mb) return;
-    int r = __ldg(d.rank + (jb >> 5)) + __popc(word & ((1u << sh) - 1u));
+    int r = rbase + __popc(word & ((1u << sh) - 1u));
 #pragma unroll
     for (int k = 0; k < kVec; ++k) {
         if (mb & (1u << k)) {
@@ -384,21 +505,34 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x / P.trials, t = blockIdx.x % P.trials;
-    if (!index_matches(P)) return;                 // kernel 1 has reported it
     const float* rec = P.rec + (long long)row * kRecFloats;
     const int nseg = C * kCW, Lw = Ls / kCW;
+    // everything that does not depend on the record's sums is requested up front
+    DrawCtx d;
+    d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
+    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
+    d.c.inv_s = __ldcg(rec + kRecInvS);
+    const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
+    const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
+    d.identity = P.header[kHdrIdentity] != 0;
+    if (!index_matches(P)) return;                 // kernel 1 has reported it
 
     if (warp == 0) {   // prefix sums over the segments, fp64
-        double iw[2], ir[2], ip[2];
+        constexpr int Q = kMaxSeg / 32;
+        double iw[Q], ir[Q], ip[Q];
+        double cw = 0.0, cr = 0.0, cp = 0.0;
         float alpha_l = 0.f;
 #pragma unroll
-        for (int it = 0; it < 2; ++it) {
+        for (int it = 0; it < Q; ++it) {
             const int s = lane + 32 * it;
             iw[it] = ir[it] = ip[it] = 0.0;
             if (s < nseg) {
                 const float4 v = __ldcg(reinterpret_cast<const float4*>(rec + 16) + s);
                 iw[it] = (double)v.x; alpha_l += v.y; ir[it] = (double)v.z; ip[it] = (double)v.w;
             }
+        }
+#pragma unroll
+        for (int it = 0; it < Q; ++it) {
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const double a = __shfl_up_sync(0xffffffffu, iw[it], o);
@@ -406,12 +540,10 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
                 const double e = __shfl_up_sync(0xffffffffu, ip[it], o);
                 if (lane >= o) { iw[it] += a; ir[it] += b; ip[it] += e; }
             }
-        }
-        iw[1] += __shfl_sync(0xffffffffu, iw[0], 31);
-        ir[1] += __shfl_sync(0xffffffffu, ir[0], 31);
-        ip[1] += __shfl_sync(0xffffffffu, ip[0], 31);
-#pragma unroll
-        for (int it = 0; it < 2; ++it) {
+            iw[it] += cw; ir[it] += cr; ip[it] += cp;
+            cw = __shfl_sync(0xffffffffu, iw[it], 31);
+            cr = __shfl_sync(0xffffffffu, ir[it], 31);
+            cp = __shfl_sync(0xffffffffu, ip[it], 31);
             const int s = lane + 32 * it;
             if (s < nseg) { cdfW[s] = iw[it]; cdfR[s] = ir[it]; cdfP[s] = ip[it]; }
         }
@@ -420,10 +552,6 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
     }
     __syncthreads();
     const double S_d = cdfW[nseg - 1], R_d = cdfR[nseg - 1], Pt_d = cdfP[nseg - 1];
-    DrawCtx d;
-    d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
-    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
-    d.c.inv_s = __ldcg(rec + kRecInvS);
     if (t == 0 && tid == 0) {
         if (P.alpha) P.alpha[row] = alpha_s;
         if (P.theta) P.theta[row] = d.c.theta;
@@ -433,14 +561,11 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
     const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
     d.zrow = zrow; d.yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
     d.zvec = (reinterpret_cast<uintptr_t>(zrow) & 15u) == 0;
-    d.mask = P.mask; d.rank = P.rank; d.slot = P.slot; d.N = P.N; d.identity = P.header[kHdrIdentity] != 0;
+    d.mask = P.mask; d.rank = P.rank; d.slot = P.slot; d.N = P.N;
 
-    const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
-    const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
-
-    // group 0 (warps 0-7): the draft draw from w; group 1 (warps 8-15): the residual draw, computed
+    // group 0 (first half of the warps): the draft draw from w; group 1: the residual draw, computed
     // alongside (it is only used if the draft is rejected)
-    const int g = warp / kCW, wg = warp % kCW;
+    const int g = warp / kGW, wg = warp % kGW;
     const bool from_p = !(R_d > 0.0);                 // p and q~ coincide: the replacement comes from p itself
     const double* cdf = g == 0 ? cdfW : (from_p ? cdfP : cdfR);
     const int what = g == 0 ? kPickW : (from_p ? kPickP : kPickR);
@@ -450,7 +575,7 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
     const int seg_lo = (seg / kCW) * Ls + (seg % kCW) * Lw;
     const int seg_end = min(P.N, seg_lo + Lw);
     const int nch = (Lw + kSeg - 1) / kSeg;
-    for (int ch = wg; ch < nch; ch += kCW) {
+    for (int ch = wg; ch < nch; ch += kGW) {
         float p[kVec], w[kVec], x[kVec];
         draw_x<TZ, TY, KIND>(d, what, seg_lo + ch * kSeg + lane * kVec, seg_end, p, w, x);
         float s = 0.f;
@@ -475,7 +600,7 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
         if (chosen < 0) { chosen = last_pos; r_in = INFINITY; }      // rounding: the last positive token
         if (chosen < 0) {
             if (wg == 0 && lane == 0) { res_tok[g] = seg_lo; res_p[g] = 0.f; res_w[g] = 0.f; }
-        } else if (chosen % kCW == wg) {
+        } else if (chosen % kGW == wg) {
             float p[kVec], w[kVec], x[kVec];
             draw_x<TZ, TY, KIND>(d, what, seg_lo + chosen * kSeg + lane * kVec, seg_end, p, w, x);
             int sel = pick_in_segment(x, r_in, lane);
@@ -520,22 +645,26 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
 // ------------------------------------------------------------------------------------------------
 struct Geometry { int C, Ls, cap; size_t smem; };
 
-static bool plan_geometry(int N, int n, size_t es, Geometry& g) {
+static bool plan_geometry(int N, int n, size_t es, size_t ys, Geometry& g) {
     int C = 1;
     while (C < kMaxC && ((size_t)N * es + C - 1) / C > 32768) C *= 2;      // slices of at most 32 KB if 8 CTAs allow
     const int per = (N + C - 1) / C;
-    const int Ls = (per + 255) / 256 * 256;
+    const int Ls = (per + 32 * kCW - 1) / (32 * kCW) * (32 * kCW);
     const long long expect = ((long long)n * Ls + N - 1) / N;
     long long cap = expect + expect / 8 + 64;
     const long long most = n < Ls ? n : Ls;
     if (cap > most) cap = most;
     cap = (cap + 31) / 32 * 32;
     const size_t zbytes = ((size_t)Ls * es + 127) & ~size_t(127);
-    size_t smem = zbytes + (size_t)cap * sizeof(float2);
+    auto total = [&](long long k) {
+        const size_t yb = ((size_t)(k + 16) * ys + 127) & ~size_t(127);
+        return zbytes + 2 * yb + (size_t)k * 8;
+    };
+    size_t smem = total(cap);
     if (smem > 200 * 1024) {
         if (zbytes > 160 * 1024) return false;
-        cap = (long long)((200 * 1024 - zbytes) / sizeof(float2)) / 32 * 32;
-        smem = zbytes + (size_t)cap * sizeof(float2);
+        cap = (long long)((200 * 1024 - zbytes - 512) / (8 + 2 * ys)) / 32 * 32;
+        smem = total(cap);
     }
     if ((Ls / kCW + kSeg - 1) / kSeg > kMaxChunks) return false;
     g.C = C; g.Ls = Ls; g.cap = (int)cap; g.smem = smem;
@@ -548,7 +677,7 @@ static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)P.rows * g.C, 1, 1);
+    cfg.gridDim = dim3((unsigned)g.C, 1, 1);
     cfg.blockDim = dim3(kCT, 1, 1);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = s;
@@ -557,7 +686,27 @@ static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_
     attr[0].val.clusterDim.x = g.C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, kern, P, g.C, g.Ls, g.cap);
+    // how many clusters fit on the device at once (cached per kernel instance, shape and device)
+    static thread_local int c_dev = -1, c_C = 0, c_G = 0;
+    static thread_local size_t c_smem = 0;
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev != c_dev || g.C != c_C || g.smem != c_smem) {
+        int sms = 0, per_sm = 0, ncl = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kCT, g.smem);
+        if (e != cudaSuccess) return e;
+        cfg.gridDim = dim3((unsigned)(sms * per_sm / g.C * g.C), 1, 1);
+        e = cudaOccupancyMaxActiveClusters(&ncl, kern, &cfg);
+        if (e != cudaSuccess) return e;
+        if (ncl < 1) return cudaErrorNotSupported;
+        c_dev = dev; c_C = g.C; c_smem = g.smem; c_G = ncl;
+    }
+    const int G = P.rows < c_G ? P.rows : c_G;
+    cfg.gridDim = dim3((unsigned)G * g.C, 1, 1);
+    e = cudaLaunchKernelEx(&cfg, kern, P, g.C, g.Ls, g.cap, G);
     if (e != cudaSuccess) return e;
     rdk_draw_kernel<TZ, TY, KIND><<<(unsigned)(P.rows * P.trials), kDT, 0, s>>>(P, g.C, g.Ls);
     return cudaGetLastError();
@@ -579,7 +728,7 @@ cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int bat
     if ((long long)P.rows * kMaxC > 0x7fffffffLL || (long long)P.rows * P.trials > 0x7fffffffLL) return cudaErrorNotSupported;
     if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < cluster_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
     Geometry g;
-    if (!plan_geometry(P.N, P.n, es, g)) return cudaErrorNotSupported;
+    if (!plan_geometry(P.N, P.n, es, ty == RDK_F32 ? 4 : 2, g)) return cudaErrorNotSupported;
     P.rec = static_cast<float*>(ws);
     P.counters = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + idx_align((size_t)P.rows * kRecFloats * sizeof(float)));
     if (tz == RDK_F32) {

@@ -67,7 +67,7 @@ def test_argument_errors_are_reported_on_the_host(B):
     assert st == B.RDK_ERR_INVALID_ARG          # precomputed mode without w
     st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_WORKSPACE_TOO_SMALL  # the linear mode needs its workspace
-    assert L.rdk_sample_workspace_bytes(C.byref(pb), 0, 1) >= 1088 and L.rdk_sample_workspace_bytes(C.byref(pb), 1, 1) == 0
+    assert L.rdk_sample_workspace_bytes(C.byref(pb), 0, 1) >= 2112 and L.rdk_sample_workspace_bytes(C.byref(pb), 1, 1) == 0
     pb.target_dtype = 9
     st = L.rdk_sample_and_verify(C.byref(pb), 0, dummy, dummy, None, 0, dummy, 1, C.byref(out), None, 0, None)
     assert st == B.RDK_ERR_INVALID_ARG
