@@ -25,7 +25,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-WORKLOAD = "C2"
+WORKLOAD = "C2"              # default: the configuration the metric is quoted on (--workload picks another)
 N_BUFFER_SETS = 6            # distinct input batches rotated through, so every step reads HBM
 METRIC = "verified draft tokens/sec"
 UNIT = "tokens/s"
@@ -149,7 +149,9 @@ def run_reference(args):
 
     import workloads as W
     from oracle import rdk_oracle as O
-    cfg = W.CONFIGS[WORKLOAD]
+    cfg = W.CONFIGS[args.workload]
+    if cfg.path == "exact":
+        raise SystemExit("--impl reference times the benchmark's linear workloads only")
     total_steps = args.steps + args.warmup
     per_row_s = 0.04
     rows_per_step = int(max(1, min(cfg.rows, 120.0 / (per_row_s * max(1, total_steps)))))
@@ -172,17 +174,26 @@ def run_reference(args):
         step(args.warmup + i)
     dt = time.perf_counter() - t0
     value = rows_per_step * args.steps / dt
-    sample = f"{rows_per_step} row(s) of {WORKLOAD} per step through oracle.rdk_row (float64 numpy, one thread)"
+    sample = f"{rows_per_step} row(s) of {args.workload} per step through oracle.rdk_row (float64 numpy, one thread)"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: N={cfg.N} n={cfg.n} bf16 logits, linear RDK; {sample}"},
+        "config": {"workload": f"{args.workload}: N={cfg.N} n={cfg.n} bf16 logits, linear RDK; {sample}"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def _peak_tensor():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
+    return 1590.0, 1400.0, "fallback (1.59 PFLOP/s burst, earlier measurement on this pool)"
 
 
 def run_ours(args):
@@ -206,19 +217,47 @@ def run_ours(args):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
 
-    cfg = W.CONFIGS[WORKLOAD]
+    cfg = W.CONFIGS[args.workload]
+    exact = cfg.path == "exact"
     rows, trials = cfg.rows, cfg.trials
-    sets = [W.make_inputs(cfg, device=str(dev), variant=v + 100 * rank) for v in range(N_BUFFER_SETS)]
+    zb = 2 if cfg.dtype == "bf16" else 4
+    kind = B.RDK_PROBS if cfg.drafter_kind == "probs" else B.RDK_LOGITS
+    row_bytes = cfg.N * zb + cfg.n * zb + trials * 16 + 30
+    # enough distinct batches that one rotation exceeds L2 several times over (C5's operands do so alone)
+    nsets = 1 if exact else max(2, min(N_BUFFER_SETS, int(600e6 // (rows * row_bytes)) + 1))
+    sets = [W.make_inputs(cfg, device=str(dev), variant=v + 100 * rank, with_embeddings=exact and v == 0)
+            for v in range(nsets)]
     index = B.rdk_prepare_ids(sets[0]["kept_ids"], cfg.N)
-    outs = [B.alloc_outputs(rows, cfg.batch, trials, dev) for _ in range(N_BUFFER_SETS)]
+    outs = [B.alloc_outputs(rows, cfg.batch, trials, dev) for _ in range(nsets)]
     outs_nolen = [{k: v for k, v in o.items() if k != "accepted_len"} for o in outs]
-    pb = B.make_problem(index, sets[0]["target"], sets[0]["drafter"], cfg.batch, cfg.positions)
+    pb = B.make_problem(index, sets[0]["target"], sets[0]["drafter"], cfg.batch, cfg.positions, kind)
     ws = B.sample_workspace(pb, B.RDK_MODE_LINEAR, trials, dev)
 
-    def step(i, out_list=outs):
-        s = sets[i % N_BUFFER_SETS]
-        B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, s["target"], s["drafter"], None, s["uniforms"],
-                                cfg.batch, cfg.positions, out=out_list[i % N_BUFFER_SETS], ws=ws)
+    prep_ms = None
+    if exact:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        M = B.rdk_build_affinity(sets[0]["embeddings"], sets[0]["kept_ids"], cfg.tau, B.RDK_AFF_BF16_COLS)
+        e1.record()
+        torch.cuda.synchronize()
+        prep_ms = e0.elapsed_time(e1)
+        w_buf = torch.empty(rows, cfg.N, dtype=torch.float32, device=dev)
+        _, _, ews = B.rdk_redistribute_exact(index, sets[0]["drafter"], M, cfg.batch, cfg.positions, kind, w_out=w_buf)
+
+        def contraction(i):
+            B.rdk_redistribute_exact(index, sets[0]["drafter"], M, cfg.batch, cfg.positions, kind, w_out=w_buf, ws=ews)
+
+        def step(i, out_list=outs):
+            contraction(i)
+            B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, sets[0]["target"], None, w_buf, sets[0]["uniforms"],
+                                    cfg.batch, cfg.positions, kind, out=out_list[0], ws=ws)
+        launches_per_step = 3 + 2          # operand, contraction, row sums; row kernel, accepted length
+    else:
+        def step(i, out_list=outs):
+            s = sets[i % nsets]
+            B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, s["target"], s["drafter"], None, s["uniforms"],
+                                    cfg.batch, cfg.positions, kind, out=out_list[i % nsets], ws=ws)
+        launches_per_step = 2              # stream kernel, draw kernel
 
     def barrier():
         torch.cuda.synchronize()
@@ -247,31 +286,34 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     sampler.start()
     ms = timed(step, args.steps)
-    # the dominant kernel alone (no accepted-length kernel behind it), same rotation of inputs
-    ms_kernel = timed(lambda i: step(i, outs_nolen), args.steps)
+    # the dominant kernels alone: linear = stream + draw kernels (no accepted length); exact = the
+    # contraction call (operand preparation, tensor-core kernel, row sums)
+    ms_kernel = timed(contraction if exact else (lambda i: step(i, outs_nolen)), args.steps)
     sampler.stop()
     sampler.join(timeout=1.0)
     B.check_status_word(outs[0], "bench step")
 
-    # end to end: host (pinned) buffers in, host results out, copies inside the timed region
-    e2e_steps = max(3, min(args.steps, 20))
-    host_sets = []
-    for s in sets[:2]:
-        host_sets.append({k: s[k].cpu().pin_memory() for k in ("target", "drafter", "uniforms")})
-    stage = {"target": torch.empty_like(sets[0]["target"]), "drafter": torch.empty_like(sets[0]["drafter"]),
-             "uniforms": torch.empty_like(sets[0]["uniforms"]), "ws": ws}
-    host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in outs[0].items() if not k.startswith("_")}
+    e2e = None
+    if not exact:
+        # end to end: host (pinned) buffers in, host results out, copies inside the timed region
+        e2e_steps = max(3, min(args.steps, 20))
+        host_sets = [{k: s[k].cpu().pin_memory() for k in ("target", "drafter", "uniforms")} for s in sets[:2]]
+        stage = {"target": torch.empty_like(sets[0]["target"]), "drafter": torch.empty_like(sets[0]["drafter"]),
+                 "uniforms": torch.empty_like(sets[0]["uniforms"]), "ws": ws}
+        host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in outs[0].items() if not k.startswith("_")}
 
-    def e2e_step(i):
-        h = host_sets[i % len(host_sets)]
-        B.rdk_sample_and_verify_host(index, h["target"], h["drafter"], h["uniforms"], cfg.batch, cfg.positions,
-                                     stage, outs[0], host_out)
+        def e2e_step(i):
+            h = host_sets[i % len(host_sets)]
+            B.rdk_sample_and_verify_host(index, h["target"], h["drafter"], h["uniforms"], cfg.batch, cfg.positions,
+                                         stage, outs[0], host_out, kind)
 
-    for i in range(3):
-        e2e_step(i)
-    ms_e2e = timed(e2e_step, e2e_steps)
-    h2d = sum(host_sets[0][k].numel() * host_sets[0][k].element_size() for k in ("target", "drafter", "uniforms"))
-    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+        for i in range(3):
+            e2e_step(i)
+        ms_e2e = timed(e2e_step, e2e_steps)
+        h2d = sum(host_sets[0][k].numel() * host_sets[0][k].element_size() for k in ("target", "drafter", "uniforms"))
+        d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+        e2e = {"value": world * rows * trials * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps}
 
     if rank != 0:
         if dist is not None:
@@ -279,36 +321,51 @@ def run_ours(args):
         return
 
     value = world * rows * trials * args.steps / (ms * 1e-3)
-    e2e_value = world * rows * trials * e2e_steps / (ms_e2e * 1e-3)
-    peak, peak_src = _peaks()
-    zb = 2 if cfg.dtype == "bf16" else 4
-    algo_bytes = rows * (cfg.N * zb + cfg.n * zb + trials * 16 + 30)
     kernel_ms = ms_kernel / args.steps
-    achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["sources_sha256"] == _kernel_sources_hash() else None
+    if exact:
+        peak, peak_sus, peak_src = _peak_tensor()
+        flops = 2.0 * rows * cfg.n * cfg.N
+        achieved = flops / (kernel_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": None, "kernel_ms": kernel_ms, "flops_per_launch": flops, "peak_source": peak_src,
+                    "frac_of_sustained_peak": achieved / peak_sus,
+                    "kernels": "exact_operand_kernel + exact_tc_kernel + row_sum_kernel"}
+    else:
+        peak, peak_src = _peaks()
+        algo_bytes = rows * row_bytes
+        achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
+        traffic = NCU_TRAFFIC["bytes_per_launch"] if (args.workload == WORKLOAD and
+                                                      NCU_TRAFFIC["sources_sha256"] == _kernel_sources_hash()) else None
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": traffic, "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": algo_bytes,
+                    "peak_source": peak_src, "kernels": "rdk_stream_kernel + rdk_draw_kernel"}
 
-    cpu_value, cpu_dt, cpu_rows = _cpu_baseline(cfg)
+    cpu = None
+    if not args.no_cpu_baseline and not exact:
+        cpu_value, cpu_dt, cpu_rows = _cpu_baseline(cfg)
+        cpu = {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"{cpu_rows} rows of {args.workload} through oracle.rdk_row (float64 numpy, one thread, {cpu_dt:.1f} s)"}
 
+    what = ("exact RDK on tensor cores (bf16 affinity, fp32 accumulate) + sampling/verification" if exact
+            else "linear RDK (first-order redistribution + sampling/verification)")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: Llama-3-scale linear RDK, N={cfg.N}, n={cfg.n}, batch={cfg.batch}, "
-                               f"positions={cfg.positions} (rows={rows}), bf16 logits, trials={trials}",
+        "config": {"workload": f"{args.workload}: {what}, N={cfg.N}, n={cfg.n}, batch={cfg.batch}, "
+                               f"positions={cfg.positions} (rows={rows}), bf16 inputs, trials={trials}",
                    "rows_per_step": rows, "parallelism": f"replicas x{world} (no collective)",
-                   "l2": f"inputs rotate over {N_BUFFER_SETS} distinct batches "
-                         f"({N_BUFFER_SETS * algo_bytes / 1e6:.0f} MB > 126 MB L2)"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": algo_bytes,
-                     "peak_source": peak_src},
-        "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"{cpu_rows} rows of {WORKLOAD} through oracle.rdk_row "
-                                   f"(float64 numpy, one thread, {cpu_dt:.1f} s)"},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
-        "gpu_launches": 2 * args.steps,
+                   "l2": (f"operands of one step ({(cfg.N * cfg.n * 2 + rows * cfg.N * 4) / 1e6:.0f} MB) exceed the 126 MB L2"
+                          if exact else
+                          f"inputs rotate over {nsets} distinct batches ({nsets * rows * row_bytes / 1e6:.0f} MB > 126 MB L2)")},
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": e2e,
+        "gpu_launches": launches_per_step * args.steps,
         "clocks": sampler.summary(),
     }
+    if prep_ms is not None:
+        line["config"]["preprocessing_ms"] = prep_ms
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -320,6 +377,10 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=["C2", "C3", "C4", "C5"], default=WORKLOAD,
+                    help="C2 (default) is the benchmark; C3/C4 are the other linear-path sizes, C5 the exact "
+                         "tensor-core path (used for profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
