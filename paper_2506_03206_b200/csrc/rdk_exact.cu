@@ -9,7 +9,7 @@
 namespace rdk {
 
 int launch_exact_tc(const __nv_bfloat16* A, long long lda, const __nv_bfloat16* Mt, long long ldm,
-                    float* w_out, int rows, int n, int N, int32_t* status_word, cudaStream_t s);
+                    float* w_out, float* S_out, int rows, int n, int N, int32_t* status_word, cudaStream_t s);
 
 // A[r, i] = q'_{kappa_i}: soft-max over the drafter entries whose id lies in the target vocabulary
 // (Eq. tli-drafter: drop the rest, renormalise), zero for dropped entries and for the padding
@@ -195,9 +195,9 @@ extern "C" int rdk_redistribute_exact(const rdk_problem* problem, const void* dr
     }
     RDK_CUDA(cudaGetLastError());
     if (bf) {
-        st = launch_exact_tc(static_cast<const __nv_bfloat16*>(ws), lda, static_cast<const __nv_bfloat16*>(M->data), M->ld,
-                             w_out, rows, n, N, status_word, s);
-        if (st != RDK_OK) return st;
+        // the tensor-core epilogue also accumulates S (one atomic partial sum per row and tile)
+        return launch_exact_tc(static_cast<const __nv_bfloat16*>(ws), lda, static_cast<const __nv_bfloat16*>(M->data), M->ld,
+                               w_out, S_out, rows, n, N, status_word, s);
     } else {
         dim3 grid((N + 255) / 256, (rows + kSimtRows - 1) / kSimtRows);
         exact_simt_kernel<<<grid, 256, 0, s>>>(static_cast<const float*>(ws), lda, static_cast<const float*>(M->data), M->ld, w_out, rows, n, N);

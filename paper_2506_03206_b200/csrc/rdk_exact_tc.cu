@@ -30,10 +30,24 @@ constexpr int kTmemCols = 512;
 constexpr unsigned kTcSpin = 1u << 21;
 
 struct TcParams {
-    float* w; int rows, N, K;
+    float* w; float* S; int rows, N, K;
     int tiles_m, tiles_n, num_kb;
+    int full_items, num_items;       // items [0, full_items) are 256-row tiles, the rest 128-row halves
     int32_t* status_word;
 };
+
+// Work item -> first row, column tile and number of 128-row MMAs.  The last partial round of
+// 256-row tiles is cut into 128-row halves so that it costs half a round instead of a whole one.
+__device__ __forceinline__ void decode_item(const TcParams& P, int item, int& row0, int& tn, int& mt) {
+    int tile, half = -1;
+    if (item < P.full_items) tile = item;
+    else { tile = P.full_items + ((item - P.full_items) >> 1); half = (item - P.full_items) & 1; }
+    const int tm = tile % P.tiles_m;
+    tn = tile / P.tiles_m;
+    row0 = tm * kTileM + (half > 0 ? kBM : 0);
+    const int left = P.rows - row0;
+    mt = left <= 0 ? 0 : ((half < 0 && left > kBM) ? 2 : 1);
+}
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -98,7 +112,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_s;
-    const int num_items = P.tiles_m * P.tiles_n;
+    const int num_items = P.num_items;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -106,14 +120,16 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-                const int tm = item % P.tiles_m, tn = item / P.tiles_m;
+                int row0, tn, mt;
+                decode_item(P, item, row0, tn, mt);
+                if (mt == 0) continue;                                        // a half tile beyond the last row
                 for (int kb = 0; kb < P.num_kb; ++kb) {
                     if (!tc_wait(&empty_bar[stage], phase ^ 1u, abort)) { ok = false; break; }
                     unsigned char* sa = tiles + stage * kStageBytes;
                     if (lane == 0) {
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(&full_bar[stage])), "r"((uint32_t)kStageBytes) : "memory");
                     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                                 ::"r"(s32(sa)), "l"(reinterpret_cast<uint64_t>(&tmapA)), "r"(kb * kBK), "r"(tm * kTileM), "r"(s32(&full_bar[stage])) : "memory");
+                                 ::"r"(s32(sa)), "l"(reinterpret_cast<uint64_t>(&tmapA)), "r"(kb * kBK), "r"(row0), "r"(s32(&full_bar[stage])) : "memory");
                     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                                  ::"r"(s32(sa + kABytes)), "l"(reinterpret_cast<uint64_t>(&tmapB)), "r"(kb * kBK), "r"(tn * kBN), "r"(s32(&full_bar[stage])) : "memory");
                     }
@@ -128,8 +144,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
             int stage = 0; uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-                const int tm = item % P.tiles_m;
-                const int mt = (P.rows - tm * kTileM > kBM) ? 2 : 1;          // a lone 128-row remainder needs one MMA
+                int row0, tn, mt;
+                decode_item(P, item, row0, tn, mt);                           // mt = 1: a lone 128-row remainder or half
+                if (mt == 0) continue;
                 if (!tc_wait(&tmem_empty, acc_phase ^ 1u, abort)) break;      // the epilogue has drained the accumulators
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 for (int kb = 0; kb < P.num_kb; ++kb) {
@@ -166,13 +183,15 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
         const bool vec_ok = (reinterpret_cast<uintptr_t>(P.w) & 15u) == 0 && (P.N & 3) == 0;
         uint32_t acc_phase = 0;
         for (int item = blockIdx.x; item < num_items; item += gridDim.x) {
-            const int tm = item % P.tiles_m, tn = item / P.tiles_m;
-            const int mt = (P.rows - tm * kTileM > kBM) ? 2 : 1;
+            int row0, tn, mt;
+            decode_item(P, item, row0, tn, mt);
+            if (mt == 0) continue;
             if (!tc_wait(&tmem_full, acc_phase, abort)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             for (int a = 0; a < mt; ++a) {
-                const int row = tm * kTileM + a * kBM + quarter * 32 + lane;
+                const int row = row0 + a * kBM + quarter * 32 + lane;
                 float* wrow = P.w + (long long)row * P.N;
+                float rsum = 0.f;
 #pragma unroll 1
                 for (int c = 0; c < kBN / 32; ++c) {
                     uint32_t v[32];
@@ -188,6 +207,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
                         : "r"(taddr) : "memory");
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     const int col0 = tn * kBN + c * 32;
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) rsum += (col0 + q < P.N) ? __uint_as_float(v[q]) : 0.f;
                     if (row < P.rows) {
                         if (vec_ok && col0 + 32 <= P.N) {
 #pragma unroll
@@ -202,6 +223,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant
                         }
                     }
                 }
+                if (P.S && row < P.rows) atomicAdd(P.S + row, rsum);           // S = sum_j w_j, one partial per tile
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -240,7 +262,7 @@ static int make_map(EncodeTiledFn enc, CUtensorMap* map, const void* base, uint6
 }
 
 int launch_exact_tc(const __nv_bfloat16* A, long long lda, const __nv_bfloat16* Mt, long long ldm, float* w_out,
-                    int rows, int n, int N, int32_t* status_word, cudaStream_t s) {
+                    float* S_out, int rows, int n, int N, int32_t* status_word, cudaStream_t s) {
     static EncodeTiledFn enc = nullptr;
     if (!enc) {
         void* fn = nullptr;
@@ -262,7 +284,7 @@ int launch_exact_tc(const __nv_bfloat16* A, long long lda, const __nv_bfloat16* 
     st = make_map(enc, &mapB, Mt, (uint64_t)n, (uint64_t)N, (uint64_t)ldm, kBK, kBN);
     if (st != RDK_OK) return st;
     TcParams P;
-    P.w = w_out; P.rows = rows; P.N = N; P.K = n;
+    P.w = w_out; P.S = S_out; P.rows = rows; P.N = N; P.K = n;
     P.tiles_m = (rows + kTileM - 1) / kTileM;
     P.tiles_n = (N + kBN - 1) / kBN;
     P.num_kb = (n + kBK - 1) / kBK;
@@ -270,8 +292,14 @@ int launch_exact_tc(const __nv_bfloat16* A, long long lda, const __nv_bfloat16* 
     int dev = 0, sms = 0;
     RDK_CUDA(cudaGetDevice(&dev));
     RDK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const long long items = (long long)P.tiles_m * P.tiles_n;
-    const int grid = (int)(items < sms ? items : sms);
+    const long long tiles = (long long)P.tiles_m * P.tiles_n;
+    if (tiles > 0x3fffffffLL) { set_error("rdk_redistribute_exact: too many output tiles"); return RDK_ERR_UNSUPPORTED; }
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    const int rest = (int)(tiles % grid);
+    const bool split = rest > 0 && 2 * rest <= grid && tiles > grid;      // cut the last partial round into halves
+    P.full_items = split ? (int)(tiles - rest) : (int)tiles;
+    P.num_items = split ? (int)(tiles + rest) : (int)tiles;
+    if (S_out) RDK_CUDA(cudaMemsetAsync(S_out, 0, (size_t)rows * sizeof(float), s));
     const size_t smem = (size_t)kStages * kStageBytes + 1024;
     RDK_CUDA(cudaFuncSetAttribute(exact_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     exact_tc_kernel<<<grid, kTcThreads, smem, s>>>(mapA, mapB, P);
