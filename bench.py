@@ -155,7 +155,7 @@ def run_reference(args):
         raise SystemExit("--impl reference times the benchmark's linear workloads only")
     total_steps = args.steps + args.warmup
     per_row_s = 0.04
-    rows_per_step = int(max(1, min(cfg.rows, 120.0 / (per_row_s * max(1, total_steps)))))
+    rows_per_step = int(max(1, min(64, cfg.rows, 120.0 / (per_row_s * max(1, total_steps)))))
     pool = min(cfg.rows, max(rows_per_step, 16))
     inp = W.make_inputs(cfg.with_rows(pool, 1), device="cpu")
     kappa = inp["kept_ids"].numpy()
@@ -186,6 +186,21 @@ def run_reference(args):
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: the job is as fast as its slowest replica."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(rows_per_rank: int, trials: int, steps: int, world: int, ms: float) -> float:
+    """Units all ranks processed divided by the slowest rank's time (replicas: weak scaling)."""
+    return world * rows_per_rank * trials * steps / (ms * 1e-3)
 
 
 def _peak_tensor():
@@ -274,12 +289,7 @@ def run_ours(args):
             fn(i)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dist, dev)
 
     warmup = max(3, args.warmup)
     for i in range(warmup):
@@ -321,7 +331,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    value = world * rows * trials * args.steps / (ms * 1e-3)
+    value = whole_job_value(rows, trials, args.steps, world, ms)
     kernel_ms = ms_kernel / args.steps
     if exact:
         peak, peak_sus, peak_src = _peak_tensor()
