@@ -41,10 +41,6 @@ constexpr int kMaxChunks = 128;      // 256-token chunks per segment (N <= 2^21)
 // record layout (floats): 16 scalars, then 4 per segment
 enum { kRecOffg = 0, kRecInvZp, kRecYoffg, kRecInvZq, kRecTheta, kRecInvN, kRecInvS, kRecS };
 
-struct Pub1 {    // one CTA's partials; every CTA holds a copy of all C of them after the exchange
-    float m, my;
-    float E1[kCW], E2[kCW], K1[kCW], K2[kCW], Zq[kCW], th[kCW];
-};
 
 struct Scal { float offg, inv_zp, yoffg, inv_zq, theta, inv_n, inv_s; };
 
@@ -196,6 +192,20 @@ __device__ __forceinline__ YPlan plan_y(const TY* src, int kcs) {
     return p;
 }
 
+// address of `addr` (a shared-memory address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// 16-byte store into another CTA's shared memory that also counts 16 bytes on that CTA's mbarrier
+__device__ __forceinline__ void st_async_v4(uint32_t raddr, float a, float b, float c, float d, uint32_t rbar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(raddr), "f"(a), "f"(b), "f"(c), "f"(d), "r"(rbar) : "memory");
+}
+
+struct SegRec { float E1, E2, K1, K2, Zq, th, m, my; };      // one warp segment's partial sums (32 bytes)
+
 template <typename TZ, typename TY, int KIND>
 __global__ void __launch_bounds__(kCT, 2)
 rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, const int G) {
@@ -206,12 +216,11 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     TZ* zbuf = reinterpret_cast<TZ*>(dsm);
     TY* ybuf[2] = {reinterpret_cast<TY*>(dsm + zb_bytes), reinterpret_cast<TY*>(dsm + zb_bytes + yb_bytes)};
     int32_t* idsb = reinterpret_cast<int32_t*>(dsm + zb_bytes + 2 * yb_bytes);
-    float* ezb = reinterpret_cast<float*>(idsb + cap);
+    float2* ezy = reinterpret_cast<float2*>(idsb + cap);                  // (e_z, e_y) of the staged kept tokens
 
-    __shared__ Pub1 all1[2][kMaxC];        // [row parity][source CTA], written by the source CTAs
-    __shared__ float redm[kCW], redy[kCW];
+    __shared__ __align__(16) SegRec all1[2][kMaxSeg];   // [row parity][segment of the row], written by the owning CTAs
     __shared__ int rk[kCW + 1];
-    __shared__ __align__(8) unsigned long long zbar, ybar[2];
+    __shared__ __align__(8) unsigned long long zbar, ybar[2], xbar[2];
     __shared__ int fail;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -230,37 +239,48 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     const int Lw = Ls / kCW;
     const int len8 = len & ~(kVec - 1);
     const uint32_t zbytes = (uint32_t)len8 * (uint32_t)sizeof(TZ);
+    const int nseg = C * kCW;
 
     if (tid == 0) {
         fail = 0;
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&zbar)));
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&ybar[0])));
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&ybar[1])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&xbar[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&xbar[1])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid <= kCW) rk[tid] = rank_at(P, min(P.N, j0 + tid * Lw), n_valid);   // rank at the warp range borders
     for (int idx = len + tid; idx < Ls; idx += kCT) zbuf[idx] = neg_inf<TZ>();   // beyond the vocabulary: weight 0
     __syncthreads();
+    cluster.sync();                       // every CTA's barriers exist before anybody signals them
     const int r0 = rk[0];
     const int kc = rk[kCW] - r0;          // kept tokens of this slice
     const int kcs = min(kc, cap);         // ... of which this many are staged in shared memory
 
-    // Loads of one row: z slice and the drafter values of the slice's rank range.
+    // Loads of one row (z slice, drafter values of the slice's rank range), issued by the last warp:
+    // its lanes stage the few unaligned elements with plain stores, then lane 0 arms the barriers
+    // (release) and starts the bulk copies, so whoever sees a barrier complete also sees those stores.
     auto issue_loads = [&](int row, int b) {
         const TZ* zsrc = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride + j0;
         const TY* ysrc = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
-        if (tid < len - len8) zbuf[len8 + tid] = zsrc[len8 + tid];                 // ragged end of the slice
         if (identity) {
-            const YPlan yp = plan_y<TY>(ysrc + r0, kcs);
-            if (tid == kCT - 32) {
-                bulk_load(&zbar, zbuf, zsrc, zbytes);
-                bulk_load(&ybar[b], ybuf[b] + yp.sh + yp.head, ysrc + r0 + yp.head, (uint32_t)(yp.mid * sizeof(TY)));
+            if (warp == kCW - 1) {
+                const YPlan yp = plan_y<TY>(ysrc + r0, kcs);
+                if (lane < len - len8) zbuf[len8 + lane] = zsrc[len8 + lane];
+                if (lane >= 8 && lane < 8 + yp.head) { const int il = lane - 8; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
+                if (lane >= 16 && lane < 16 + yp.tail) { const int il = yp.head + yp.mid + lane - 16; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
+                __syncwarp();
+                if (lane == 0) {
+                    bulk_load(&zbar, zbuf, zsrc, zbytes);
+                    bulk_load(&ybar[b], ybuf[b] + yp.sh + yp.head, ysrc + r0 + yp.head, (uint32_t)(yp.mid * sizeof(TY)));
+                }
             }
-            if (tid >= 32 && tid < 32 + yp.head) { const int il = tid - 32; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
-            if (tid >= 64 && tid < 64 + yp.tail) { const int il = yp.head + yp.mid + tid - 64; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
         } else {
-            if (tid == kCT - 32) { bulk_load(&zbar, zbuf, zsrc, zbytes); bulk_load(&ybar[b], nullptr, nullptr, 0); }
+            if (tid < len - len8) zbuf[len8 + tid] = zsrc[len8 + tid];
             for (int il = tid; il < kcs; il += kCT) ybuf[b][il] = ysrc[__ldg(P.slot + r0 + il)];
+            __syncthreads();
+            if (tid == 0) { bulk_load(&zbar, zbuf, zsrc, zbytes); bulk_load(&ybar[b], nullptr, nullptr, 0); }
         }
     };
     auto y_shift = [&](int row) -> int {
@@ -272,12 +292,13 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     if (cid < P.rows) issue_loads(cid, 0);
     // token ids of the slice's kept tokens, in rank order: the same for every row
     for (int il = tid; il < kcs; il += kCT) idsb[il] = __ldg(P.ids + (identity ? r0 + il : __ldg(P.slot + r0 + il)));
+    __syncthreads();
 
     const int wa = warp * Lw, wb = wa + Lw;
     const int rw0 = rk[warp] - r0, rw1 = rk[warp + 1] - r0;
     const int rw1s = min(rw1, kcs);       // staged part of the warp's kept tokens
-    const int nseg = C * kCW;
     const float inv_n = 1.f / (float)P.N;
+    const uint32_t xbytes = (uint32_t)nseg * (uint32_t)sizeof(SegRec);
 
     int it = 0;
     for (int row = cid; row < P.rows; row += G, ++it) {
@@ -285,37 +306,34 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         const TY* yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
         const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
         const TY* yb = ybuf[b] + y_shift(row);
+        if (tid == 0)   // this row's exchange: nseg records of 32 bytes will arrive from the cluster
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&xbar[b])), "r"(xbytes) : "memory");
         mbar_wait(&zbar, (uint32_t)(it & 1), &fail);
         mbar_wait(&ybar[b], (uint32_t)((it >> 1) & 1), &fail);
-        __syncthreads();                  // the few elements staged with plain stores are visible
 
-        // ---- maxima of the slice's logits and of its drafter values ---------------------------------
+        // ---- this warp's maxima: its token range and the drafter values of its kept tokens ---------
         MaxAcc<TZ> mz;
         for (int cs = wa; cs < wb; cs += kSeg) {
             const int jl = cs + lane * kVec;
             if (jl < wb) mz.push(zbuf, jl);
         }
-        float my_t = -INFINITY;
+        float my_w = -INFINITY;
         if (KIND == RDK_LOGITS) {
-            for (int il = tid; il < kcs; il += kCT) my_t = fmaxf(my_t, to_float<TY>(yb[il]));
-            for (int il = cap + tid; il < kc; il += kCT)
-                my_t = fmaxf(my_t, to_float<TY>(yrow[identity ? r0 + il : __ldg(P.slot + r0 + il)]));
+            for (int il = rw0 + lane; il < rw1s; il += 32) my_w = fmaxf(my_w, to_float<TY>(yb[il]));
+            for (int il = max(rw0, cap) + lane; il < rw1; il += 32)
+                my_w = fmaxf(my_w, to_float<TY>(yrow[identity ? r0 + il : __ldg(P.slot + r0 + il)]));
+            my_w = warp_max(my_w);
+        } else {
+            my_w = 0.f;
         }
-        const float mz_w = warp_max(mz.result());
-        my_t = warp_max(my_t);
-        if (lane == 0) { redm[warp] = mz_w; redy[warp] = my_t; }
-        __syncthreads();
-        float m_c = redm[0], my_c = redy[0];
-#pragma unroll
-        for (int k = 1; k < kCW; ++k) { m_c = fmaxf(m_c, redm[k]); my_c = fmaxf(my_c, redy[k]); }
-        if (KIND == RDK_PROBS) my_c = 0.f;
+        const float m_w = warp_max(mz.result());
 
         // ---- soft-max sweep: sum e and sum e^2 over the warp's token range ----------------------------
-        const float zoff_c = -m_c * kLog2e, yoff_c = -my_c * kLog2e;
+        const float zoff_w = -m_w * kLog2e, yoff_w = -my_w * kLog2e;
         float E1 = 0.f, E2 = 0.f;
-        if (m_c > -INFINITY) {
+        if (m_w > -INFINITY) {
             float2 e1 = make_float2(0.f, 0.f), e2 = make_float2(0.f, 0.f);
-            const float2 sc = make_float2(kLog2e, kLog2e), of = make_float2(zoff_c, zoff_c);
+            const float2 sc = make_float2(kLog2e, kLog2e), of = make_float2(zoff_w, zoff_w);
 #pragma unroll 2
             for (int cs = wa; cs < wb; cs += kSeg) {
                 const int jl = cs + lane * kVec;
@@ -323,78 +341,81 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
             }
             E1 = e1.x + e1.y; E2 = e2.x + e2.y;
         }
-        // ---- kept tokens of the warp's range: e_z (cached), e_y, their sums -----------------------------
+        // ---- kept tokens of the warp's range: e_z, e_y (cached), their sums -----------------------------
         float K1 = 0.f, K2 = 0.f, Zq = 0.f, th = 0.f;
-#pragma unroll 2
+#pragma unroll 4
         for (int il = rw0 + lane; il < rw1s; il += 32) {
-            const float ez = ex2(fmaf(to_float<TZ>(zbuf[idsb[il] - j0]), kLog2e, zoff_c));
+            const float ez = ex2(fmaf(to_float<TZ>(zbuf[idsb[il] - j0]), kLog2e, zoff_w));
             const float y = to_float<TY>(yb[il]);
-            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_w)) : y;
             K1 += ez; K2 = fmaf(ez, ez, K2); Zq += ey; th = fmaf(ez, ey, th);
-            ezb[il] = ez;
+            ezy[il] = make_float2(ez, ey);
         }
         for (int il = max(rw0, cap) + lane; il < rw1; il += 32) {      // kept tokens that did not fit the cache
             const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
-            const float ez = ex2(fmaf(to_float<TZ>(zbuf[__ldg(P.ids + i) - j0]), kLog2e, zoff_c));
+            const float ez = ex2(fmaf(to_float<TZ>(zbuf[__ldg(P.ids + i) - j0]), kLog2e, zoff_w));
             const float y = to_float<TY>(yrow[i]);
-            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_w)) : y;
             K1 += ez; K2 = fmaf(ez, ez, K2); Zq += ey; th = fmaf(ez, ey, th);
         }
         E1 = warp_sum(E1); E2 = warp_sum(E2); K1 = warp_sum(K1); K2 = warp_sum(K2);
         Zq = warp_sum(Zq); th = warp_sum(th);
-        // push this warp's sums into every CTA of the cluster (lane c writes to CTA c)
+        // push this warp's record into every CTA of the cluster (lane c writes to CTA c)
         if (lane < C) {
-            Pub1* rp = cluster.map_shared_rank(&all1[b][crank], lane);
-            rp->E1[warp] = E1; rp->E2[warp] = E2; rp->K1[warp] = K1; rp->K2[warp] = K2; rp->Zq[warp] = Zq; rp->th[warp] = th;
-            if (warp == 0) { rp->m = m_c; rp->my = my_c; }
+            const uint32_t raddr = mapa_u32(smem_u32(&all1[b][crank * kCW + warp]), (uint32_t)lane);
+            const uint32_t rbar = mapa_u32(smem_u32(&xbar[b]), (uint32_t)lane);
+            st_async_v4(raddr, E1, E2, K1, K2, rbar);
+            st_async_v4(raddr + 16, Zq, th, m_w, my_w, rbar);
         }
         __syncthreads();                  // every warp is done with zbuf: the next row may stream in
-        cluster.barrier_arrive();
         if (row + G < P.rows) issue_loads(row + G, b ^ 1);
-        cluster.barrier_wait();                                                // the one exchange per row
+        mbar_wait(&xbar[b], (uint32_t)((it >> 1) & 1), &fail);                 // all nseg records have arrived
 
-        // ---- combine the C partials: every warp does it for itself, in the same order everywhere ----
+        // ---- combine the records: every warp does it for itself, in the same order everywhere ---------
         Scal c;
         float fz, fy, segA_w = 0.f, segP_w = 0.f, S_row;
         {
-            float mc = -INFINITY, myc = -INFINITY;
-            if (lane < C) { mc = all1[b][lane].m; myc = all1[b][lane].my; }
-            const float m = warp_max(mc), my = warp_max(myc);
-            const float f_l = mc > -INFINITY ? ex2((mc - m) * kLog2e) : 0.f;
-            const float g_l = myc > -INFINITY ? ex2((myc - my) * kLog2e) : 0.f;
-            float e1[kMaxSeg / 32], e2[kMaxSeg / 32], k1[kMaxSeg / 32], k2[kMaxSeg / 32];
-            float tZp = 0.f, tE2 = 0.f, tZq = 0.f, tTh = 0.f;
+            float e1[kMaxSeg / 32], e2[kMaxSeg / 32], k1[kMaxSeg / 32], k2[kMaxSeg / 32], zq[kMaxSeg / 32], tt[kMaxSeg / 32];
+            float ms[kMaxSeg / 32], mys[kMaxSeg / 32];
+            float m = -INFINITY, my = -INFINITY;
 #pragma unroll
             for (int q = 0; q < kMaxSeg / 32; ++q) {
                 const int s = lane + 32 * q;
-                const bool valid = s < nseg;
-                const int cc = valid ? s / kCW : 0, w = s % kCW;
-                const float f = __shfl_sync(0xffffffffu, f_l, cc), g = __shfl_sync(0xffffffffu, g_l, cc);
-                e1[q] = e2[q] = k1[q] = k2[q] = 0.f;
-                if (valid) {
-                    const Pub1* rp = &all1[b][cc];
-                    e1[q] = f * rp->E1[w]; e2[q] = f * f * rp->E2[w];
-                    k1[q] = f * rp->K1[w]; k2[q] = f * f * rp->K2[w];
-                    tZp += e1[q]; tE2 += e2[q];
-                    tZq += g * rp->Zq[w]; tTh += f * g * rp->th[w];
+                e1[q] = e2[q] = k1[q] = k2[q] = zq[q] = tt[q] = 0.f; ms[q] = mys[q] = -INFINITY;
+                if (s < nseg) {
+                    const float4 u = *reinterpret_cast<const float4*>(&all1[b][s]);
+                    const float4 v = *(reinterpret_cast<const float4*>(&all1[b][s]) + 1);
+                    e1[q] = u.x; e2[q] = u.y; k1[q] = u.z; k2[q] = u.w; zq[q] = v.x; tt[q] = v.y; ms[q] = v.z; mys[q] = v.w;
                 }
+                m = fmaxf(m, ms[q]); my = fmaxf(my, mys[q]);
+            }
+            m = warp_max(m); my = warp_max(my);
+            float tZp = 0.f, tE2 = 0.f, tZq = 0.f, tTh = 0.f, f_q[kMaxSeg / 32], g_q[kMaxSeg / 32];
+#pragma unroll
+            for (int q = 0; q < kMaxSeg / 32; ++q) {
+                const float f = ms[q] > -INFINITY ? ex2((ms[q] - m) * kLog2e) : 0.f;
+                const float g = mys[q] > -INFINITY ? ex2((mys[q] - my) * kLog2e) : 0.f;
+                f_q[q] = f; g_q[q] = g;
+                e1[q] *= f; e2[q] *= f * f; k1[q] *= f; k2[q] *= f * f;
+                tZp += e1[q]; tE2 += e2[q]; tZq += g * zq[q]; tTh += f * g * tt[q];
             }
             tZp = warp_sum(tZp); tE2 = warp_sum(tE2); tZq = warp_sum(tZq); tTh = warp_sum(tTh);
             const float inv_zp = 1.f / tZp, inv_zq = 1.f / tZq;
             const float theta = tTh * inv_zp * inv_zq;
             const float P2 = tE2 * inv_zp * inv_zp;
             S_row = fmaf(-theta * P2 * inv_n, inv_n, 1.f);           // 1 - theta sum p^2 / N^2 (next term below 1/N^2)
-            // this warp's own segment: total p mass, and sum over its not-kept tokens of p / (N + p)
+            // this warp's own segment: total p mass, sum over its not-kept tokens of p / (N + p), scales
             const int s_me = crank * kCW + warp;
+            float f_me = 0.f, g_me = 0.f;
 #pragma unroll
             for (int q = 0; q < kMaxSeg / 32; ++q) {
                 const float Po = fmaxf(0.f, e1[q] - k1[q]) * inv_zp;
                 const float P2o = fmaxf(0.f, e2[q] - k2[q]) * inv_zp * inv_zp;
                 const float pa = e1[q] * inv_zp, aa = inv_n * (Po - inv_n * P2o);
                 const float pb_ = __shfl_sync(0xffffffffu, pa, s_me & 31), ab_ = __shfl_sync(0xffffffffu, aa, s_me & 31);
-                if ((s_me >> 5) == q) { segP_w = pb_; segA_w = ab_; }
+                const float fb_ = __shfl_sync(0xffffffffu, f_q[q], s_me & 31), gb_ = __shfl_sync(0xffffffffu, g_q[q], s_me & 31);
+                if ((s_me >> 5) == q) { segP_w = pb_; segA_w = ab_; f_me = fb_; g_me = gb_; }
             }
-            const float f_me = __shfl_sync(0xffffffffu, f_l, crank), g_me = __shfl_sync(0xffffffffu, g_l, crank);
             c.offg = -m * kLog2e; c.inv_zp = inv_zp; c.yoffg = -my * kLog2e; c.inv_zq = inv_zq; c.theta = theta;
             c.inv_n = inv_n; c.inv_s = 1.f / S_row;
             fz = f_me * inv_zp; fy = (KIND == RDK_LOGITS ? g_me : 1.f) * inv_zq;
@@ -402,18 +423,17 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
 
         // ---- kept tokens again: sum of min(p, q~) --------------------------------------------------
         float ak = 0.f;
-#pragma unroll 2
+#pragma unroll 4
         for (int il = rw0 + lane; il < rw1s; il += 32) {
-            const float y = to_float<TY>(yb[il]);
-            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
-            const float p = ezb[il] * fz;
-            ak += fminf(p, taylor_w(c, p, ey * fy) * c.inv_s);
+            const float2 v = ezy[il];
+            const float p = v.x * fz;
+            ak += fminf(p, taylor_w(c, p, v.y * fy) * c.inv_s);
         }
         for (int il = max(rw0, cap) + lane; il < rw1; il += 32) {
             const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
-            const float ez = ex2(fmaf(to_float<TZ>(zrow[__ldg(P.ids + i)]), kLog2e, zoff_c));
+            const float ez = ex2(fmaf(to_float<TZ>(zrow[__ldg(P.ids + i)]), kLog2e, zoff_w));
             const float y = to_float<TY>(yrow[i]);
-            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_c)) : y;
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_w)) : y;
             const float p = ez * fz;
             ak += fminf(p, taylor_w(c, p, ey * fy) * c.inv_s);
         }
@@ -440,7 +460,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         }
     }
     if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
-    cluster.sync();                        // remote shared memory must outlive its readers
+    cluster.sync();                        // no CTA leaves while others may still write into it
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -658,12 +678,12 @@ static bool plan_geometry(int N, int n, size_t es, size_t ys, Geometry& g) {
     const size_t zbytes = ((size_t)Ls * es + 127) & ~size_t(127);
     auto total = [&](long long k) {
         const size_t yb = ((size_t)(k + 16) * ys + 127) & ~size_t(127);
-        return zbytes + 2 * yb + (size_t)k * 8;
+        return zbytes + 2 * yb + (size_t)k * 12;
     };
     size_t smem = total(cap);
     if (smem > 200 * 1024) {
         if (zbytes > 160 * 1024) return false;
-        cap = (long long)((200 * 1024 - zbytes - 512) / (8 + 2 * ys)) / 32 * 32;
+        cap = (long long)((200 * 1024 - zbytes - 512) / (12 + 2 * ys)) / 32 * 32;
         smem = total(cap);
     }
     if ((Ls / kCW + kSeg - 1) / kSeg > kMaxChunks) return false;
