@@ -30,7 +30,7 @@ namespace rdk {
 
 constexpr int kCT = 256;             // threads per CTA of kernel 1
 constexpr int kCW = kCT / 32;        // warps per CTA; each owns a contiguous token range = one segment
-constexpr int kMaxC = 8;             // portable cluster size
+constexpr int kMaxC = 8;             // the portable cluster size (16-CTA clusters were tried: fewer resident CTAs, no gain)
 constexpr int kMaxSeg = kMaxC * kCW;
 constexpr int kMinClusterN = 4096;
 constexpr unsigned kSpinLimit = 1u << 22;
@@ -665,9 +665,9 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
 // ------------------------------------------------------------------------------------------------
 struct Geometry { int C, Ls, cap; size_t smem; };
 
-static bool plan_geometry(int N, int n, size_t es, size_t ys, Geometry& g) {
+static bool plan_geometry(int N, int n, size_t es, size_t ys, int max_c, Geometry& g) {
     int C = 1;
-    while (C < kMaxC && ((size_t)N * es + C - 1) / C > 32768) C *= 2;      // slices of at most 32 KB if 8 CTAs allow
+    while (C < max_c && ((size_t)N * es + C - 1) / C > 32768) C *= 2;      // slices of at most 32 KB if 8 CTAs allow
     const int per = (N + C - 1) / C;
     const int Ls = (per + 32 * kCW - 1) / (32 * kCW) * (32 * kCW);
     const long long expect = ((long long)n * Ls + N - 1) / N;
@@ -696,6 +696,10 @@ static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_
     auto kern = rdk_stream_kernel<TZ, TY, KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
     if (e != cudaSuccess) return e;
+    if (g.C > 8) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)g.C, 1, 1);
     cfg.blockDim = dim3(kCT, 1, 1);
@@ -747,16 +751,18 @@ cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int bat
     if ((reinterpret_cast<uintptr_t>(P.target) & 15u) || ((P.target_stride * (long long)es) & 15)) return cudaErrorNotSupported;
     if ((long long)P.rows * kMaxC > 0x7fffffffLL || (long long)P.rows * P.trials > 0x7fffffffLL) return cudaErrorNotSupported;
     if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < cluster_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
-    Geometry g;
-    if (!plan_geometry(P.N, P.n, es, ty == RDK_F32 ? 4 : 2, g)) return cudaErrorNotSupported;
     P.rec = static_cast<float*>(ws);
     P.counters = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + idx_align((size_t)P.rows * kRecFloats * sizeof(float)));
-    if (tz == RDK_F32) {
-        if (ty == RDK_F32) return launch_kind_c<float, float>(P, kind, g, s);
-        return launch_kind_c<float, __nv_bfloat16>(P, kind, g, s);
+    cudaError_t e = cudaErrorNotSupported;
+    for (int max_c = kMaxC; max_c >= 8 && e == cudaErrorNotSupported; max_c /= 2) {   // 16-CTA clusters first, then 8
+        Geometry g;
+        if (!plan_geometry(P.N, P.n, es, ty == RDK_F32 ? 4 : 2, max_c, g)) continue;
+        if (tz == RDK_F32) e = ty == RDK_F32 ? launch_kind_c<float, float>(P, kind, g, s) : launch_kind_c<float, __nv_bfloat16>(P, kind, g, s);
+        else e = ty == RDK_F32 ? launch_kind_c<__nv_bfloat16, float>(P, kind, g, s) : launch_kind_c<__nv_bfloat16, __nv_bfloat16>(P, kind, g, s);
+        if (g.C <= 8) break;
+        if (e != cudaSuccess && e != cudaErrorNotSupported) { (void)cudaGetLastError(); e = cudaErrorNotSupported; }   // 16 not schedulable here
     }
-    if (ty == RDK_F32) return launch_kind_c<__nv_bfloat16, float>(P, kind, g, s);
-    return launch_kind_c<__nv_bfloat16, __nv_bfloat16>(P, kind, g, s);
+    return e;
 }
 
 }  // namespace rdk
