@@ -207,7 +207,7 @@ __device__ __forceinline__ void st_async_v4(uint32_t raddr, float a, float b, fl
 struct SegRec { float E1, E2, K1, K2, Zq, th, m, my; };      // one warp segment's partial sums (32 bytes)
 
 template <typename TZ, typename TY, int KIND>
-__global__ void __launch_bounds__(kCT, 2)
+__global__ void __launch_bounds__(kCT, 3)
 rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, const int G) {
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(128) unsigned char dsm[];
@@ -233,6 +233,8 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     }
     const bool identity = P.header[kHdrIdentity] != 0;
     const int n_valid = P.header[kHdrValid];
+    // the draw kernel may be scheduled already; it waits for this whole grid before reading the records
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int j0 = crank * Ls;
     const int len = max(0, min(P.N - j0, Ls));
@@ -527,15 +529,15 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
     const int row = blockIdx.x / P.trials, t = blockIdx.x % P.trials;
     const float* rec = P.rec + (long long)row * kRecFloats;
     const int nseg = C * kCW, Lw = Ls / kCW;
-    // everything that does not depend on the record's sums is requested up front
     DrawCtx d;
-    d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
-    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
-    d.c.inv_s = __ldcg(rec + kRecInvS);
     const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
     const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
     d.identity = P.header[kHdrIdentity] != 0;
     if (!index_matches(P)) return;                 // kernel 1 has reported it
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // kernel 1 (launched just before) is complete and visible
+    d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
+    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
+    d.c.inv_s = __ldcg(rec + kRecInvS);
 
     if (warp == 0) {   // prefix sums over the segments, fp64
         constexpr int Q = kMaxSeg / 32;
@@ -732,8 +734,17 @@ static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_
     cfg.gridDim = dim3((unsigned)G * g.C, 1, 1);
     e = cudaLaunchKernelEx(&cfg, kern, P, g.C, g.Ls, g.cap, G);
     if (e != cudaSuccess) return e;
-    rdk_draw_kernel<TZ, TY, KIND><<<(unsigned)(P.rows * P.trials), kDT, 0, s>>>(P, g.C, g.Ls);
-    return cudaGetLastError();
+    cudaLaunchConfig_t dcfg = {};
+    dcfg.gridDim = dim3((unsigned)(P.rows * P.trials), 1, 1);
+    dcfg.blockDim = dim3(kDT, 1, 1);
+    dcfg.dynamicSmemBytes = 0;
+    dcfg.stream = s;
+    cudaLaunchAttribute dattr[1];
+    dattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while kernel 1 drains
+    dattr[0].val.programmaticStreamSerializationAllowed = 1;
+    dcfg.attrs = dattr;
+    dcfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&dcfg, rdk_draw_kernel<TZ, TY, KIND>, P, g.C, g.Ls);
 }
 
 template <typename TZ, typename TY>
