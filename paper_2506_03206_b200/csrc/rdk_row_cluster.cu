@@ -218,6 +218,8 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     int32_t* idsb = reinterpret_cast<int32_t*>(dsm + zb_bytes + 2 * yb_bytes);
     float2* ezy = reinterpret_cast<float2*>(idsb + cap);                  // (e_z, e_y) of the staged kept tokens
 
+    __shared__ __align__(16) float4 segv[kCW];
+    __shared__ float bcs[8];
     __shared__ __align__(16) SegRec all1[2][kMaxSeg];   // [row parity][segment of the row], written by the owning CTAs
     __shared__ int rk[kCW + 1];
     __shared__ __align__(8) unsigned long long zbar, ybar[2], xbar[2];
@@ -373,10 +375,8 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         if (row + G < P.rows) issue_loads(row + G, b ^ 1);
         mbar_wait(&xbar[b], (uint32_t)((it >> 1) & 1), &fail);                 // all nseg records have arrived
 
-        // ---- combine the records: every warp does it for itself, in the same order everywhere ---------
-        Scal c;
-        float fz, fy, segA_w = 0.f, segP_w = 0.f, S_row;
-        {
+        // ---- combine the records (warp 0), hand every warp its scalars through shared memory --------
+        if (warp == 0) {
             float e1[kMaxSeg / 32], e2[kMaxSeg / 32], k1[kMaxSeg / 32], k2[kMaxSeg / 32], zq[kMaxSeg / 32], tt[kMaxSeg / 32];
             float ms[kMaxSeg / 32], mys[kMaxSeg / 32];
             float m = -INFINITY, my = -INFINITY;
@@ -392,36 +392,38 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
                 m = fmaxf(m, ms[q]); my = fmaxf(my, mys[q]);
             }
             m = warp_max(m); my = warp_max(my);
-            float tZp = 0.f, tE2 = 0.f, tZq = 0.f, tTh = 0.f, f_q[kMaxSeg / 32], g_q[kMaxSeg / 32];
+            float tZp = 0.f, tZq = 0.f, tTh = 0.f, f_q[kMaxSeg / 32], g_q[kMaxSeg / 32];
 #pragma unroll
             for (int q = 0; q < kMaxSeg / 32; ++q) {
                 const float f = ms[q] > -INFINITY ? ex2((ms[q] - m) * kLog2e) : 0.f;
                 const float g = mys[q] > -INFINITY ? ex2((mys[q] - my) * kLog2e) : 0.f;
                 f_q[q] = f; g_q[q] = g;
                 e1[q] *= f; e2[q] *= f * f; k1[q] *= f; k2[q] *= f * f;
-                tZp += e1[q]; tE2 += e2[q]; tZq += g * zq[q]; tTh += f * g * tt[q];
+                tZp += e1[q]; tZq += g * zq[q]; tTh += f * g * tt[q];
             }
-            tZp = warp_sum(tZp); tE2 = warp_sum(tE2); tZq = warp_sum(tZq); tTh = warp_sum(tTh);
+            tZp = warp_sum(tZp); tZq = warp_sum(tZq); tTh = warp_sum(tTh);
             const float inv_zp = 1.f / tZp, inv_zq = 1.f / tZq;
             const float theta = tTh * inv_zp * inv_zq;
-            const float P2 = tE2 * inv_zp * inv_zp;
-            S_row = fmaf(-theta * P2 * inv_n, inv_n, 1.f);           // 1 - theta sum p^2 / N^2 (next term below 1/N^2)
-            // this warp's own segment: total p mass, sum over its not-kept tokens of p / (N + p), scales
-            const int s_me = crank * kCW + warp;
-            float f_me = 0.f, g_me = 0.f;
+            // own segments: total p mass, sum over the not-kept tokens of p / (N + p), scales
 #pragma unroll
             for (int q = 0; q < kMaxSeg / 32; ++q) {
-                const float Po = fmaxf(0.f, e1[q] - k1[q]) * inv_zp;
-                const float P2o = fmaxf(0.f, e2[q] - k2[q]) * inv_zp * inv_zp;
-                const float pa = e1[q] * inv_zp, aa = inv_n * (Po - inv_n * P2o);
-                const float pb_ = __shfl_sync(0xffffffffu, pa, s_me & 31), ab_ = __shfl_sync(0xffffffffu, aa, s_me & 31);
-                const float fb_ = __shfl_sync(0xffffffffu, f_q[q], s_me & 31), gb_ = __shfl_sync(0xffffffffu, g_q[q], s_me & 31);
-                if ((s_me >> 5) == q) { segP_w = pb_; segA_w = ab_; f_me = fb_; g_me = gb_; }
+                const int s = lane + 32 * q;
+                if (s < nseg && s / kCW == crank) {
+                    const float Po = fmaxf(0.f, e1[q] - k1[q]) * inv_zp;
+                    const float P2o = fmaxf(0.f, e2[q] - k2[q]) * inv_zp * inv_zp;
+                    segv[s % kCW] = make_float4(e1[q] * inv_zp, inv_n * (Po - inv_n * P2o), f_q[q] * inv_zp,
+                                                (KIND == RDK_LOGITS ? g_q[q] : 1.f) * inv_zq);
+                }
             }
-            c.offg = -m * kLog2e; c.inv_zp = inv_zp; c.yoffg = -my * kLog2e; c.inv_zq = inv_zq; c.theta = theta;
-            c.inv_n = inv_n; c.inv_s = 1.f / S_row;
-            fz = f_me * inv_zp; fy = (KIND == RDK_LOGITS ? g_me : 1.f) * inv_zq;
+            if (lane == 0) { bcs[0] = -m * kLog2e; bcs[1] = inv_zp; bcs[2] = -my * kLog2e; bcs[3] = inv_zq; bcs[4] = theta; }
         }
+        __syncthreads();
+        Scal c;
+        c.offg = bcs[0]; c.inv_zp = bcs[1]; c.yoffg = bcs[2]; c.inv_zq = bcs[3]; c.theta = bcs[4];
+        c.inv_n = inv_n; c.inv_s = 1.f;      // S = 1 - theta sum p^2 / N^2 + ... rounds to 1 in fp32 for N >= 4096 (|S - 1| < 2^-24)
+        const float S_row = 1.f;
+        const float4 sv = segv[warp];
+        const float segP_w = sv.x, segA_w = sv.y, fz = sv.z, fy = sv.w;
 
         // ---- kept tokens again: sum of min(p, q~) --------------------------------------------------
         float ak = 0.f;
