@@ -28,10 +28,9 @@ namespace cg = cooperative_groups;
 
 namespace rdk {
 
-constexpr int kCT = 256;             // threads per CTA of kernel 1
-constexpr int kCW = kCT / 32;        // warps per CTA; each owns a contiguous token range = one segment
+constexpr int kMaxCW = 16;           // warps (= segments) per CTA of kernel 1: 8 or 16
 constexpr int kMaxC = 8;             // the portable cluster size (16-CTA clusters were tried: fewer resident CTAs, no gain)
-constexpr int kMaxSeg = kMaxC * kCW;
+constexpr int kMaxSeg = kMaxC * kMaxCW;
 constexpr int kMinClusterN = 4096;
 constexpr unsigned kSpinLimit = 1u << 22;
 constexpr int kDT = 256;             // threads per CTA of kernel 2: 4 warps for the draft, 4 for the residual
@@ -206,9 +205,11 @@ __device__ __forceinline__ void st_async_v4(uint32_t raddr, float a, float b, fl
 
 struct SegRec { float E1, E2, K1, K2, Zq, th, m, my; };      // one warp segment's partial sums (32 bytes)
 
-template <typename TZ, typename TY, int KIND>
-__global__ void __launch_bounds__(kCT, 3)
+template <typename TZ, typename TY, int KIND, int CT>
+__global__ void __launch_bounds__(CT, CT == 256 ? 3 : 1)
 rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, const int G) {
+    constexpr int CW = CT / 32;          // warps per CTA; each owns a contiguous token range = one segment
+    constexpr int MAXSEG = kMaxC * CW;
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(128) unsigned char dsm[];
     const size_t zb_bytes = ((size_t)Ls * sizeof(TZ) + 127) & ~size_t(127);
@@ -218,10 +219,10 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     int32_t* idsb = reinterpret_cast<int32_t*>(dsm + zb_bytes + 2 * yb_bytes);
     float2* ezy = reinterpret_cast<float2*>(idsb + cap);                  // (e_z, e_y) of the staged kept tokens
 
-    __shared__ __align__(16) float4 segv[kCW];
+    __shared__ __align__(16) float4 segv[CW];
     __shared__ float bcs[8];
-    __shared__ __align__(16) SegRec all1[2][kMaxSeg];   // [row parity][segment of the row], written by the owning CTAs
-    __shared__ int rk[kCW + 1];
+    __shared__ __align__(16) SegRec all1[2][MAXSEG];   // [row parity][segment of the row], written by the owning CTAs
+    __shared__ int rk[CW + 1];
     __shared__ __align__(8) unsigned long long zbar, ybar[2], xbar[2];
     __shared__ int fail;
 
@@ -240,10 +241,10 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
 
     const int j0 = crank * Ls;
     const int len = max(0, min(P.N - j0, Ls));
-    const int Lw = Ls / kCW;
+    const int Lw = Ls / CW;
     const int len8 = len & ~(kVec - 1);
     const uint32_t zbytes = (uint32_t)len8 * (uint32_t)sizeof(TZ);
-    const int nseg = C * kCW;
+    const int nseg = C * CW;
 
     if (tid == 0) {
         fail = 0;
@@ -254,12 +255,12 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&xbar[1])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (tid <= kCW) rk[tid] = rank_at(P, min(P.N, j0 + tid * Lw), n_valid);   // rank at the warp range borders
-    for (int idx = len + tid; idx < Ls; idx += kCT) zbuf[idx] = neg_inf<TZ>();   // beyond the vocabulary: weight 0
+    if (tid <= CW) rk[tid] = rank_at(P, min(P.N, j0 + tid * Lw), n_valid);   // rank at the warp range borders
+    for (int idx = len + tid; idx < Ls; idx += CT) zbuf[idx] = neg_inf<TZ>();   // beyond the vocabulary: weight 0
     __syncthreads();
     cluster.sync();                       // every CTA's barriers exist before anybody signals them
     const int r0 = rk[0];
-    const int kc = rk[kCW] - r0;          // kept tokens of this slice
+    const int kc = rk[CW] - r0;          // kept tokens of this slice
     const int kcs = min(kc, cap);         // ... of which this many are staged in shared memory
 
     // Loads of one row (z slice, drafter values of the slice's rank range), issued by the last warp:
@@ -269,7 +270,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         const TZ* zsrc = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride + j0;
         const TY* ysrc = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
         if (identity) {
-            if (warp == kCW - 1) {
+            if (warp == CW - 1) {
                 const YPlan yp = plan_y<TY>(ysrc + r0, kcs);
                 if (lane < len - len8) zbuf[len8 + lane] = zsrc[len8 + lane];
                 if (lane >= 8 && lane < 8 + yp.head) { const int il = lane - 8; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
@@ -282,7 +283,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
             }
         } else {
             if (tid < len - len8) zbuf[len8 + tid] = zsrc[len8 + tid];
-            for (int il = tid; il < kcs; il += kCT) ybuf[b][il] = ysrc[__ldg(P.slot + r0 + il)];
+            for (int il = tid; il < kcs; il += CT) ybuf[b][il] = ysrc[__ldg(P.slot + r0 + il)];
             __syncthreads();
             if (tid == 0) { bulk_load(&zbar, zbuf, zsrc, zbytes); bulk_load(&ybar[b], nullptr, nullptr, 0); }
         }
@@ -295,7 +296,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
 
     if (cid < P.rows) issue_loads(cid, 0);
     // token ids of the slice's kept tokens, in rank order: the same for every row
-    for (int il = tid; il < kcs; il += kCT) idsb[il] = __ldg(P.ids + (identity ? r0 + il : __ldg(P.slot + r0 + il)));
+    for (int il = tid; il < kcs; il += CT) idsb[il] = __ldg(P.ids + (identity ? r0 + il : __ldg(P.slot + r0 + il)));
     __syncthreads();
 
     const int wa = warp * Lw, wb = wa + Lw;
@@ -366,7 +367,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         Zq = warp_sum(Zq); th = warp_sum(th);
         // push this warp's record into every CTA of the cluster (lane c writes to CTA c)
         if (lane < C) {
-            const uint32_t raddr = mapa_u32(smem_u32(&all1[b][crank * kCW + warp]), (uint32_t)lane);
+            const uint32_t raddr = mapa_u32(smem_u32(&all1[b][crank * CW + warp]), (uint32_t)lane);
             const uint32_t rbar = mapa_u32(smem_u32(&xbar[b]), (uint32_t)lane);
             st_async_v4(raddr, E1, E2, K1, K2, rbar);
             st_async_v4(raddr + 16, Zq, th, m_w, my_w, rbar);
@@ -377,11 +378,11 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
 
         // ---- combine the records (warp 0), hand every warp its scalars through shared memory --------
         if (warp == 0) {
-            float e1[kMaxSeg / 32], e2[kMaxSeg / 32], k1[kMaxSeg / 32], k2[kMaxSeg / 32], zq[kMaxSeg / 32], tt[kMaxSeg / 32];
-            float ms[kMaxSeg / 32], mys[kMaxSeg / 32];
+            float e1[MAXSEG / 32], e2[MAXSEG / 32], k1[MAXSEG / 32], k2[MAXSEG / 32], zq[MAXSEG / 32], tt[MAXSEG / 32];
+            float ms[MAXSEG / 32], mys[MAXSEG / 32];
             float m = -INFINITY, my = -INFINITY;
 #pragma unroll
-            for (int q = 0; q < kMaxSeg / 32; ++q) {
+            for (int q = 0; q < MAXSEG / 32; ++q) {
                 const int s = lane + 32 * q;
                 e1[q] = e2[q] = k1[q] = k2[q] = zq[q] = tt[q] = 0.f; ms[q] = mys[q] = -INFINITY;
                 if (s < nseg) {
@@ -392,9 +393,9 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
                 m = fmaxf(m, ms[q]); my = fmaxf(my, mys[q]);
             }
             m = warp_max(m); my = warp_max(my);
-            float tZp = 0.f, tZq = 0.f, tTh = 0.f, f_q[kMaxSeg / 32], g_q[kMaxSeg / 32];
+            float tZp = 0.f, tZq = 0.f, tTh = 0.f, f_q[MAXSEG / 32], g_q[MAXSEG / 32];
 #pragma unroll
-            for (int q = 0; q < kMaxSeg / 32; ++q) {
+            for (int q = 0; q < MAXSEG / 32; ++q) {
                 const float f = ms[q] > -INFINITY ? ex2((ms[q] - m) * kLog2e) : 0.f;
                 const float g = mys[q] > -INFINITY ? ex2((mys[q] - my) * kLog2e) : 0.f;
                 f_q[q] = f; g_q[q] = g;
@@ -406,12 +407,12 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
             const float theta = tTh * inv_zp * inv_zq;
             // own segments: total p mass, sum over the not-kept tokens of p / (N + p), scales
 #pragma unroll
-            for (int q = 0; q < kMaxSeg / 32; ++q) {
+            for (int q = 0; q < MAXSEG / 32; ++q) {
                 const int s = lane + 32 * q;
-                if (s < nseg && s / kCW == crank) {
+                if (s < nseg && s / CW == crank) {
                     const float Po = fmaxf(0.f, e1[q] - k1[q]) * inv_zp;
                     const float P2o = fmaxf(0.f, e2[q] - k2[q]) * inv_zp * inv_zp;
-                    segv[s % kCW] = make_float4(e1[q] * inv_zp, inv_n * (Po - inv_n * P2o), f_q[q] * inv_zp,
+                    segv[s % CW] = make_float4(e1[q] * inv_zp, inv_n * (Po - inv_n * P2o), f_q[q] * inv_zp,
                                                 (KIND == RDK_LOGITS ? g_q[q] : 1.f) * inv_zq);
                 }
             }
@@ -452,7 +453,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
             const float Kw = fy * Zq - fy * xs * th + c.theta * (xs * K1 - xs * xs * K2);
             const float oov = c.theta * segA_w;
             const float a_s = oov * c.inv_s + ak;
-            reinterpret_cast<float4*>(rec + 16)[crank * kCW + warp] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP_w - a_s), segP_w);
+            reinterpret_cast<float4*>(rec + 16)[crank * CW + warp] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP_w - a_s), segP_w);
         }
         if (crank == 0) {
             if (tid == 0) {
@@ -460,7 +461,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
                 rec[kRecTheta] = c.theta; rec[kRecInvN] = c.inv_n; rec[kRecInvS] = c.inv_s; rec[kRecS] = S_row;
             }
             if (P.counters && row % P.positions == 0)
-                for (int t = tid; t < P.trials; t += kCT) P.counters[(row / P.positions) * P.trials + t] = 0;
+                for (int t = tid; t < P.trials; t += CT) P.counters[(row / P.positions) * P.trials + t] = 0;
         }
     }
     if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
@@ -520,7 +521,7 @@ __device__ __forceinline__ void draw_x(const DrawCtx& d, int what, int jb, int s
 
 template <typename TZ, typename TY, int KIND>
 __global__ void __launch_bounds__(kDT)
-rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
+rdk_draw_kernel(const RowParams P, const int C, const int Ls, const int cw) {
     __shared__ double cdfW[kMaxSeg], cdfR[kMaxSeg], cdfP[kMaxSeg];
     __shared__ float sums[2][kMaxChunks];
     __shared__ float alpha_s;
@@ -530,7 +531,7 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x / P.trials, t = blockIdx.x % P.trials;
     const float* rec = P.rec + (long long)row * kRecFloats;
-    const int nseg = C * kCW, Lw = Ls / kCW;
+    const int nseg = C * cw, Lw = Ls / cw;
     DrawCtx d;
     const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
     const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
@@ -596,7 +597,7 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
     const double thr = g == 0 ? (double)u0 * S_d : (double)u2 * (from_p ? Pt_d : R_d);
     const int seg = min(first_above(cdf, nseg, thr), nseg - 1);
     const float rem = (float)(thr - (seg ? cdf[seg - 1] : 0.0));
-    const int seg_lo = (seg / kCW) * Ls + (seg % kCW) * Lw;
+    const int seg_lo = (seg / cw) * Ls + (seg % cw) * Lw;
     const int seg_end = min(P.N, seg_lo + Lw);
     const int nch = (Lw + kSeg - 1) / kSeg;
     for (int ch = wg; ch < nch; ch += kGW) {
@@ -667,9 +668,10 @@ rdk_draw_kernel(const RowParams P, const int C, const int Ls) {
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-struct Geometry { int C, Ls, cap; size_t smem; };
+struct Geometry { int C, Ls, cap, ct; size_t smem; };
 
-static bool plan_geometry(int N, int n, size_t es, size_t ys, int max_c, Geometry& g) {
+static bool plan_geometry(int N, int n, size_t es, size_t ys, int max_c, int ct, Geometry& g) {
+    const int kCW = ct / 32;
     int C = 1;
     while (C < max_c && ((size_t)N * es + C - 1) / C > 32768) C *= 2;      // slices of at most 32 KB if 8 CTAs allow
     const int per = (N + C - 1) / C;
@@ -691,13 +693,14 @@ static bool plan_geometry(int N, int n, size_t es, size_t ys, int max_c, Geometr
         smem = total(cap);
     }
     if ((Ls / kCW + kSeg - 1) / kSeg > kMaxChunks) return false;
-    g.C = C; g.Ls = Ls; g.cap = (int)cap; g.smem = smem;
+    g.C = C; g.Ls = Ls; g.cap = (int)cap; g.smem = smem; g.ct = ct;
     return true;
 }
 
-template <typename TZ, typename TY, int KIND>
-static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_t s) {
-    auto kern = rdk_stream_kernel<TZ, TY, KIND>;
+template <typename TZ, typename TY, int KIND, int CT>
+static cudaError_t launch_ct(const RowParams& P, const Geometry& g, cudaStream_t s) {
+    constexpr int kCT = CT;
+    auto kern = rdk_stream_kernel<TZ, TY, KIND, CT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
     if (e != cudaSuccess) return e;
     if (g.C > 8) {
@@ -746,7 +749,12 @@ static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_
     dattr[0].val.programmaticStreamSerializationAllowed = 1;
     dcfg.attrs = dattr;
     dcfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&dcfg, rdk_draw_kernel<TZ, TY, KIND>, P, g.C, g.Ls);
+    return cudaLaunchKernelEx(&dcfg, rdk_draw_kernel<TZ, TY, KIND>, P, g.C, g.Ls, CT / 32);
+}
+
+template <typename TZ, typename TY, int KIND>
+static cudaError_t launch_one(const RowParams& P, const Geometry& g, cudaStream_t s) {
+    return g.ct == 256 ? launch_ct<TZ, TY, KIND, 256>(P, g, s) : launch_ct<TZ, TY, KIND, 512>(P, g, s);
 }
 
 template <typename TZ, typename TY>
@@ -769,7 +777,9 @@ cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int bat
     cudaError_t e = cudaErrorNotSupported;
     for (int max_c = kMaxC; max_c >= 8 && e == cudaErrorNotSupported; max_c /= 2) {   // 16-CTA clusters first, then 8
         Geometry g;
-        if (!plan_geometry(P.N, P.n, es, ty == RDK_F32 ? 4 : 2, max_c, g)) continue;
+        if (!plan_geometry(P.N, P.n, es, ty == RDK_F32 ? 4 : 2, max_c, 256, g)) continue;
+        // a slice so large that only one CTA fits per SM gets 16 warps instead of 8
+        if (g.smem > 110 * 1024 && !plan_geometry(P.N, P.n, es, ty == RDK_F32 ? 4 : 2, max_c, 512, g)) continue;
         if (tz == RDK_F32) e = ty == RDK_F32 ? launch_kind_c<float, float>(P, kind, g, s) : launch_kind_c<float, __nv_bfloat16>(P, kind, g, s);
         else e = ty == RDK_F32 ? launch_kind_c<__nv_bfloat16, float>(P, kind, g, s) : launch_kind_c<__nv_bfloat16, __nv_bfloat16>(P, kind, g, s);
         if (g.C <= 8) break;
