@@ -28,6 +28,7 @@ namespace cg = cooperative_groups;
 
 namespace rdk {
 
+constexpr int kKeptPerLane = 24;     // kept tokens per lane whose ids stay in registers (768 per warp)
 constexpr int kMaxCW = 16;           // warps (= segments) per CTA of kernel 1: 8 or 16
 constexpr int kMaxC = 8;             // the portable cluster size (16-CTA clusters were tried: fewer resident CTAs, no gain)
 constexpr int kMaxSeg = kMaxC * kMaxCW;
@@ -216,8 +217,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     const size_t yb_bytes = ((size_t)(cap + 16) * sizeof(TY) + 127) & ~size_t(127);
     TZ* zbuf = reinterpret_cast<TZ*>(dsm);
     TY* ybuf[2] = {reinterpret_cast<TY*>(dsm + zb_bytes), reinterpret_cast<TY*>(dsm + zb_bytes + yb_bytes)};
-    int32_t* idsb = reinterpret_cast<int32_t*>(dsm + zb_bytes + 2 * yb_bytes);
-    float2* ezy = reinterpret_cast<float2*>(idsb + cap);                  // (e_z, e_y) of the staged kept tokens
+    float* ezb = reinterpret_cast<float*>(dsm + zb_bytes + 2 * yb_bytes);   // e_z of the staged kept tokens
 
     __shared__ __align__(16) float4 segv[CW];
     __shared__ float bcs[8];
@@ -295,13 +295,21 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     };
 
     if (cid < P.rows) issue_loads(cid, 0);
-    // token ids of the slice's kept tokens, in rank order: the same for every row
-    for (int il = tid; il < kcs; il += CT) idsb[il] = __ldg(P.ids + (identity ? r0 + il : __ldg(P.slot + r0 + il)));
     __syncthreads();
 
     const int wa = warp * Lw, wb = wa + Lw;
     const int rw0 = rk[warp] - r0, rw1 = rk[warp + 1] - r0;
-    const int rw1s = min(rw1, kcs);       // staged part of the warp's kept tokens
+    const int rw1s = max(rw0, min(min(rw1, kcs), rw0 + 32 * kKeptPerLane));   // part of the warp's kept tokens handled from registers / shared memory
+    // local token index of this lane's kept tokens (lane + 32 k -th of the warp's range): the same for
+    // every row, so they live in registers, two 16-bit indices per word
+    uint32_t idr[kKeptPerLane / 2];
+#pragma unroll
+    for (int k = 0; k < kKeptPerLane; ++k) {
+        const int il = rw0 + lane + 32 * k;
+        uint32_t v = 0;
+        if (il < rw1s) v = (uint32_t)(__ldg(P.ids + (identity ? r0 + il : __ldg(P.slot + r0 + il))) - j0);
+        if (k & 1) idr[k / 2] |= v << 16; else idr[k / 2] = v;
+    }
     const float inv_n = 1.f / (float)P.N;
     const uint32_t xbytes = (uint32_t)nseg * (uint32_t)sizeof(SegRec);
 
@@ -325,7 +333,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         float my_w = -INFINITY;
         if (KIND == RDK_LOGITS) {
             for (int il = rw0 + lane; il < rw1s; il += 32) my_w = fmaxf(my_w, to_float<TY>(yb[il]));
-            for (int il = max(rw0, cap) + lane; il < rw1; il += 32)
+            for (int il = rw1s + lane; il < rw1; il += 32)
                 my_w = fmaxf(my_w, to_float<TY>(yrow[identity ? r0 + il : __ldg(P.slot + r0 + il)]));
             my_w = warp_max(my_w);
         } else {
@@ -348,15 +356,20 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         }
         // ---- kept tokens of the warp's range: e_z, e_y (cached), their sums -----------------------------
         float K1 = 0.f, K2 = 0.f, Zq = 0.f, th = 0.f;
-#pragma unroll 4
-        for (int il = rw0 + lane; il < rw1s; il += 32) {
-            const float ez = ex2(fmaf(to_float<TZ>(zbuf[idsb[il] - j0]), kLog2e, zoff_w));
-            const float y = to_float<TY>(yb[il]);
-            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_w)) : y;
-            K1 += ez; K2 = fmaf(ez, ez, K2); Zq += ey; th = fmaf(ez, ey, th);
-            ezy[il] = make_float2(ez, ey);
+#pragma unroll
+        for (int k = 0; k < kKeptPerLane; ++k) {
+            if (rw0 + 32 * k >= rw1s) break;                      // warp-uniform
+            const int il = rw0 + lane + 32 * k;
+            if (il < rw1s) {
+                const uint32_t jl = (k & 1) ? (idr[k / 2] >> 16) : (idr[k / 2] & 0xffffu);
+                const float ez = ex2(fmaf(to_float<TZ>(zbuf[jl]), kLog2e, zoff_w));
+                const float y = to_float<TY>(yb[il]);
+                const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_w)) : y;
+                K1 += ez; K2 = fmaf(ez, ez, K2); Zq += ey; th = fmaf(ez, ey, th);
+                ezb[il] = ez;
+            }
         }
-        for (int il = max(rw0, cap) + lane; il < rw1; il += 32) {      // kept tokens that did not fit the cache
+        for (int il = rw1s + lane; il < rw1; il += 32) {               // kept tokens beyond the staged part
             const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
             const float ez = ex2(fmaf(to_float<TZ>(zbuf[__ldg(P.ids + i) - j0]), kLog2e, zoff_w));
             const float y = to_float<TY>(yrow[i]);
@@ -430,11 +443,12 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         float ak = 0.f;
 #pragma unroll 4
         for (int il = rw0 + lane; il < rw1s; il += 32) {
-            const float2 v = ezy[il];
-            const float p = v.x * fz;
-            ak += fminf(p, taylor_w(c, p, v.y * fy) * c.inv_s);
+            const float y = to_float<TY>(yb[il]);
+            const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_w)) : y;
+            const float p = ezb[il] * fz;
+            ak += fminf(p, taylor_w(c, p, ey * fy) * c.inv_s);
         }
-        for (int il = max(rw0, cap) + lane; il < rw1; il += 32) {
+        for (int il = rw1s + lane; il < rw1; il += 32) {
             const int i = identity ? r0 + il : __ldg(P.slot + r0 + il);
             const float ez = ex2(fmaf(to_float<TZ>(zrow[__ldg(P.ids + i)]), kLog2e, zoff_w));
             const float y = to_float<TY>(yrow[i]);
@@ -684,15 +698,15 @@ static bool plan_geometry(int N, int n, size_t es, size_t ys, int max_c, int ct,
     const size_t zbytes = ((size_t)Ls * es + 127) & ~size_t(127);
     auto total = [&](long long k) {
         const size_t yb = ((size_t)(k + 16) * ys + 127) & ~size_t(127);
-        return zbytes + 2 * yb + (size_t)k * 12;
+        return zbytes + 2 * yb + (size_t)k * 4;
     };
     size_t smem = total(cap);
     if (smem > 200 * 1024) {
         if (zbytes > 160 * 1024) return false;
-        cap = (long long)((200 * 1024 - zbytes - 512) / (12 + 2 * ys)) / 32 * 32;
+        cap = (long long)((200 * 1024 - zbytes - 512) / (4 + 2 * ys)) / 32 * 32;
         smem = total(cap);
     }
-    if ((Ls / kCW + kSeg - 1) / kSeg > kMaxChunks) return false;
+    if ((Ls / kCW + kSeg - 1) / kSeg > kMaxChunks || Ls > 65536) return false;   // local token indices are 16-bit
     g.C = C; g.Ls = Ls; g.cap = (int)cap; g.smem = smem; g.ct = ct;
     return true;
 }
