@@ -96,37 +96,51 @@ rdk_row_kernel(const RowParams P) {
     float sq = 0.f;
     for (int tile = 0; tile < P.num_tiles; ++tile) {
         const int base = tile * kTile + c.tid * kVec;
-        if (base >= P.N) break;
-        float z[kVec], e[kVec];
-        load8<TZ>(zrow, base, P.N, c.zvec, -INFINITY, z);
-        float vmax = z[0];
+        if (MODE == RDK_MODE_LINEAR && base >= P.N) break;
+        float wsum_t = 0.f;
+        if (base < P.N) {
+            if (MODE == RDK_MODE_PRECOMPUTED_W) {       // w does not depend on the soft-max: its sums ride along
+                float w8[kVec];
+                load8<float>(wrow, base, P.N, c.wvec, 0.f, w8);
 #pragma unroll
-        for (int k = 1; k < kVec; ++k) vmax = fmaxf(vmax, z[k]);
-        if (vmax == -INFINITY) continue;
-        if (vmax > zs.m) {
-            const float sc = ex2((zs.m - vmax) * kLog2e);
-            zs.s *= sc; zs.b *= sc; zs.m = vmax;
-        }
-        const float off = -zs.m * kLog2e;
+                for (int k = 0; k < kVec; ++k) wsum_t += w8[k];
+            }
+            float z[kVec], e[kVec];
+            load8<TZ>(zrow, base, P.N, c.zvec, -INFINITY, z);
+            float vmax = z[0];
 #pragma unroll
-        for (int k = 0; k < kVec; ++k) { e[k] = ex2(fmaf(z[k], kLog2e, off)); zs.s += e[k]; }
-        if (MODE == RDK_MODE_LINEAR) {
-            const uint32_t word = __ldg(P.mask + (base >> 5));
-            const int sh = base & 31;
-            const uint32_t mb = (word >> sh) & 0xffu;
-            if (mb) {
-                int r = __ldg(P.rank + (base >> 5)) + __popc(word & ((1u << sh) - 1u));
+            for (int k = 1; k < kVec; ++k) vmax = fmaxf(vmax, z[k]);
+            if (vmax > -INFINITY) {
+                if (vmax > zs.m) {
+                    const float sc = ex2((zs.m - vmax) * kLog2e);
+                    zs.s *= sc; zs.b *= sc; zs.m = vmax;
+                }
+                const float off = -zs.m * kLog2e;
 #pragma unroll
-                for (int k = 0; k < kVec; ++k) {
-                    if (mb & (1u << k)) {
-                        const int i = c.identity ? r : __ldg(P.slot + r);
-                        ++r;
-                        const float y = to_float<TY>(yrow[i]);
-                        if (KIND == RDK_LOGITS) { ms_push(ys, y); ms_push(ts, z[k] + y); }
-                        else { sq += y; zs.b += e[k] * y; }
+                for (int k = 0; k < kVec; ++k) { e[k] = ex2(fmaf(z[k], kLog2e, off)); zs.s += e[k]; }
+                if (MODE == RDK_MODE_LINEAR) {
+                    const uint32_t word = __ldg(P.mask + (base >> 5));
+                    const int sh = base & 31;
+                    const uint32_t mb = (word >> sh) & 0xffu;
+                    if (mb) {
+                        int r = __ldg(P.rank + (base >> 5)) + __popc(word & ((1u << sh) - 1u));
+#pragma unroll
+                        for (int k = 0; k < kVec; ++k) {
+                            if (mb & (1u << k)) {
+                                const int i = c.identity ? r : __ldg(P.slot + r);
+                                ++r;
+                                const float y = to_float<TY>(yrow[i]);
+                                if (KIND == RDK_LOGITS) { ms_push(ys, y); ms_push(ts, z[k] + y); }
+                                else { sq += y; zs.b += e[k] * y; }
+                            }
+                        }
                     }
                 }
             }
+        }
+        if (MODE == RDK_MODE_PRECOMPUTED_W) {
+            wsum_t = warp_sum(wsum_t);
+            if (c.lane == 0) seg_w[tile * kRowWarps + c.warp] = wsum_t;
         }
     }
     zs = ms_warp(zs);
@@ -163,8 +177,8 @@ rdk_row_kernel(const RowParams P) {
     c.inv_zq = 1.f / bc[3];
     c.theta = bc[4];
 
-    // ---- pass 2: S = sum_j w_j and the per-segment sums of w ------------------------------------
-    for (int tile = 0; tile < P.num_tiles; ++tile) {
+    // ---- pass 2: S = sum_j w_j and the per-segment sums of w (done in pass 1 for a given w) -------
+    for (int tile = 0; MODE == RDK_MODE_LINEAR && tile < P.num_tiles; ++tile) {
         const int base = tile * kTile + c.tid * kVec;
         float sum = 0.f;
         if (base < P.N) {
