@@ -47,6 +47,7 @@ Pins (tests/test_oracle_pins.py, `-m "not gpu"`), per function:
                      q~_t a_t + (1 - alpha) r_t = p_t for every t (output distributed as p);
                      Lemma 2.3 alpha = 1 - ||k||_1 = 1 - 0.5 ||p - q~||_1; Monte-Carlo
   accepted_len       brute force over all accept patterns
+  emit_sequence      brute force over all accept patterns; bonus draw frequency against p
 """
 from __future__ import annotations
 
@@ -256,6 +257,23 @@ def accepted_len(accepted: np.ndarray) -> np.ndarray:
             k += 1
         out[b] = k
     return out
+
+
+# ----------------------------------------------------------------------------------------------
+# O10  the emitted sequence (Algorithm 4 steps 7-9): the accepted drafts d_1..d_j followed by one
+#      more token t: the residual draw made where the first rejection happened, or, if every draft
+#      was accepted, a fresh draw t ~ p from the target row that follows the last draft
+# ----------------------------------------------------------------------------------------------
+def emit_sequence(draft, accepted, out_token, p_bonus, u_bonus) -> list:
+    """draft, accepted, out_token: per draft position of ONE sequence (out_token[k] is the residual
+    draw of position k where it was rejected).  p_bonus: target distribution after all drafts.
+    Returns [d_1, ..., d_j, t] (length j + 1, between 1 and positions + 1)."""
+    positions = len(draft)
+    j = 0
+    while j < positions and bool(accepted[j]):
+        j += 1
+    t = int(out_token[j]) if j < positions else inverse_cdf(p_bonus, u_bonus)
+    return [int(d) for d in draft[:j]] + [t]
 
 
 # ----------------------------------------------------------------------------------------------

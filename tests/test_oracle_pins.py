@@ -425,3 +425,24 @@ def test_accepted_len_bruteforce():
                 want += 1
             assert g == want
             assert g == (P if row.all() else int(np.argmin(row)))
+
+
+# ---------------------------------------------------------------- emitted sequence (O10)
+def test_emit_sequence_bruteforce_and_bonus_distribution():
+    rng = np.random.default_rng(15)
+    p_bonus = _rand_dist(rng, 6)
+    for P in [1, 2, 4]:
+        draft = rng.integers(0, 100, size=P)
+        resid = rng.integers(100, 200, size=P)
+        for pat in itertools.product([False, True], repeat=P):
+            seq = O.emit_sequence(draft, pat, resid, p_bonus, 0.5)
+            j = P if all(pat) else list(pat).index(False)
+            assert len(seq) == j + 1 and seq[:j] == draft[:j].tolist()          # between 1 and P + 1 tokens
+            if j < P:
+                assert seq[-1] == resid[j]                                      # the residual draw of the first rejection
+            else:
+                assert seq[-1] == O.inverse_cdf(p_bonus, 0.5) and 0 <= seq[-1] < 6
+    # when every draft is accepted the extra token is distributed as p
+    u = rng.uniform(size=30000)
+    counts = np.bincount([O.emit_sequence([7], [True], [9], p_bonus, x)[-1] for x in u], minlength=6)
+    assert np.abs(counts / u.size - p_bonus).max() < 0.012
