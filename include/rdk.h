@@ -218,6 +218,27 @@ int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* 
                           void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * rdk_emit_sequences -- Algorithm 4 steps 7-9: what each sequence emits after verification.  For
+ * sequence b and trial t, with j = number of leading accepted positions:
+ *   seq_tokens[b, t, 0..j) = the accepted drafts d_1..d_j,
+ *   seq_tokens[b, t, j]    = out_token of position j (the residual draw of the first rejection) if
+ *                            j < positions, else a draw t ~ softmax(bonus_target[b]) -- the target
+ *                            distribution after all drafts -- by inverse CDF with uniform lane 3 of
+ *                            the sequence's last position,
+ *   seq_len[b, t]          = j + 1  (between 1 and positions + 1).
+ *   bonus_target  device [batch, N] target logits of problem->target_dtype, row stride in elements
+ *                 (0 means N)
+ *   uniforms, draft_token, accepted, out_token: as given to / produced by rdk_sample_and_verify
+ *   seq_tokens    device int32 [batch, trials, positions + 1] (entries beyond seq_len are untouched)
+ *   seq_len       device int32 [batch, trials]
+ * Only problem->N, batch, positions and target_dtype are read.
+ * ------------------------------------------------------------------------------------------- */
+int rdk_emit_sequences(const rdk_problem* problem, const void* bonus_target, int64_t bonus_row_stride,
+                       const float* uniforms, int32_t trials, const int32_t* draft_token,
+                       const uint8_t* accepted, const int32_t* out_token, int32_t* seq_tokens,
+                       int32_t* seq_len, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * rdk_sample_and_verify_host -- the same step (linear mode) for callers whose logits live in HOST
  * memory: copies target_host / drafter_host / uniforms_host to the caller's device staging
  * buffers, runs rdk_sample_and_verify, copies the per-(row, trial) and per-row results back and

@@ -29,7 +29,7 @@ EXPORTS = [
     "rdk_version", "rdk_status_string", "rdk_last_error", "rdk_kept_index_bytes", "rdk_prepare_ids",
     "rdk_build_affinity_workspace_bytes", "rdk_build_affinity", "rdk_exact_workspace_bytes",
     "rdk_redistribute_exact", "rdk_redistribute_exact_static", "rdk_redistribute_linear",
-    "rdk_sample_workspace_bytes", "rdk_sample_and_verify",
+    "rdk_sample_workspace_bytes", "rdk_sample_and_verify", "rdk_emit_sequences",
     "rdk_sample_and_verify_host",
 ]
 
@@ -100,6 +100,9 @@ def lib() -> C.CDLL:
                                             C.POINTER(rdk_outputs), C.c_void_p, C.c_size_t, C.c_void_p]
         L.rdk_sample_workspace_bytes.restype = C.c_size_t
         L.rdk_sample_workspace_bytes.argtypes = [C.POINTER(rdk_problem), C.c_int32, C.c_int32]
+        L.rdk_emit_sequences.restype = C.c_int
+        L.rdk_emit_sequences.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.c_int64, C.c_void_p, C.c_int32,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.rdk_sample_and_verify_host.restype = C.c_int
         L.rdk_sample_and_verify_host.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.c_void_p, C.c_void_p,
                                                  C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -311,6 +314,22 @@ def rdk_sample_and_verify(index: KeptIndex, mode: int, target: torch.Tensor,
                                        C.byref(o), ws.data_ptr(), ws.numel(), _stream()), "rdk_sample_and_verify")
     out["_ws"] = ws        # keep the workspace alive until the stream has consumed it
     return out
+
+
+def rdk_emit_sequences(N: int, batch: int, positions: int, bonus_target: torch.Tensor, uniforms: torch.Tensor,
+                       draft_token: torch.Tensor, accepted: torch.Tensor, out_token: torch.Tensor):
+    """Returns (seq_tokens int32 [batch, trials, positions + 1], seq_len int32 [batch, trials])."""
+    _rows2d(bonus_target, "bonus_target")
+    trials = uniforms.numel() // (batch * positions * 4)
+    pb = rdk_problem()
+    pb.N, pb.n, pb.batch, pb.positions = N, 1, batch, positions
+    pb.target_dtype = _dtype_code(bonus_target)
+    seq = torch.full((batch, trials, positions + 1), -1, dtype=torch.int32, device=bonus_target.device)
+    ln = torch.empty(batch, trials, dtype=torch.int32, device=bonus_target.device)
+    _check(lib().rdk_emit_sequences(C.byref(pb), bonus_target.data_ptr(), bonus_target.stride(0), uniforms.data_ptr(),
+                                    trials, draft_token.data_ptr(), accepted.data_ptr(), out_token.data_ptr(),
+                                    seq.data_ptr(), ln.data_ptr(), _stream()), "rdk_emit_sequences")
+    return seq, ln
 
 
 def rdk_sample_and_verify_host(index: KeptIndex, target_host: torch.Tensor, drafter_host: torch.Tensor,
