@@ -208,3 +208,34 @@ def test_full_size_configs_sampled_rows(name, nrows):
     mean_alpha = a.mean().item()
     sigma = (a * (1 - a)).sum().sqrt().item() / cfg.rows
     assert abs(acc.double().mean().item() - mean_alpha) < 5 * sigma + 1e-3
+
+
+def test_extreme_pruning_heavy_tailed_logits_and_tli_baseline():
+    """200k vocabulary, 500 kept tokens, Student-t logits (the shape of the paper's synthetic
+    experiment): parity of the linear path on sampled rows, and the TLI baseline (q~ = q', obtained by
+    handing the sampler w = q' scattered to the full vocabulary) next to it."""
+    rdk = _rdk()
+    B = rdk.binding
+    cfg = W.CONFIGS["T1"]
+    inp = W.make_inputs(cfg, device="cuda")
+    rows = [0, 17, 63, cfg.rows - 1]
+    _run_linear(cfg, inp, rows=rows, check_qtilde=False).assert_ok(max_ambiguous_frac=0.25)
+    idx = rdk.rdk_prepare_ids(inp["kept_ids"], cfg.N)
+    out_rdk = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, inp["target"], inp["drafter"], None, inp["uniforms"],
+                                        cfg.batch, cfg.positions)
+    # TLI: q' placed at the kept ids, zero elsewhere (generator-side scatter of the drafter soft-max)
+    qp = torch.softmax(inp["drafter"].float(), dim=-1)
+    w = torch.zeros(cfg.rows, cfg.N, dtype=torch.float32, device="cuda")
+    w[:, inp["kept_ids"].long()] = qp
+    out_tli = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_PRECOMPUTED_W, inp["target"], None, w, inp["uniforms"],
+                                        cfg.batch, cfg.positions)
+    torch.cuda.synchronize()
+    kappa = inp["kept_ids"].cpu().numpy()
+    for r in rows:
+        p = O.softmax(W.to_f64(inp["target"][r]))
+        q_tli = O.tli_project(W.to_f64(w[r])[kappa], kappa, cfg.N)
+        assert abs(float(out_tli["alpha"][r]) - O.acceptance_rate(p, q_tli)) < PU.ABS_TOL
+    a_rdk, a_tli = out_rdk["alpha"].double(), out_tli["alpha"].double()
+    # the first-order formula moves only about theta / N of the mass: both rates agree to ~1e-5 here
+    assert torch.all((a_rdk - a_tli).abs() < 1e-4)
+    print("T1 mean alpha: RDK(linear)", a_rdk.mean().item(), "TLI", a_tli.mean().item())

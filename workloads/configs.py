@@ -39,6 +39,7 @@ class RDKConfig:
     drafter_kind: str = "logits"   # "logits" | "probs"
     tau: float = 0.1
     seed: int = 20250603
+    noise: str = "normal"          # "normal" | "student_t5" (heavy-tailed logits, Sec. 5.1 "Logits")
 
     @property
     def rows(self) -> int:
@@ -65,6 +66,12 @@ CONFIGS: Dict[str, RDKConfig] = {
     "C4": RDKConfig("C4", N=262144, n=32768, batch=512, positions=4, dtype="bf16", path="linear",
                     kept_rule="zipf", sigma=3.0, zipf_bias=True, rho=0.7, emb_dim=512, trials=1,
                     seed=104),
+    # Shape of the paper's synthetic acceptance experiment (Sec. 5.2): a 200k vocabulary pruned to 500
+    # kept tokens, heavy-tailed (Student-t, 5 degrees of freedom) logits.  Not one of the benchmark
+    # configurations; used for parity at extreme pruning and to report RDK next to TLI.
+    "T1": RDKConfig("T1", N=200000, n=500, batch=32, positions=4, dtype="bf16", path="linear",
+                    kept_rule="zipf", sigma=3.0, zipf_bias=True, rho=0.8, emb_dim=64, trials=1,
+                    seed=106, noise="student_t5"),
     # Dense exact redistribution on tensor cores.
     "C5": RDKConfig("C5", N=32768, n=8192, batch=1024, positions=1, dtype="bf16", path="exact",
                     kept_rule="uniform", sigma=2.0, zipf_bias=False, rho=0.8, emb_dim=128, trials=1,
@@ -147,10 +154,19 @@ def make_inputs(cfg: RDKConfig, device: str = "cpu", variant: int = 0,
     target = torch.empty(rows, N, dtype=dt, device=dev)
     drafter = torch.empty(rows, n, dtype=dt, device=dev)
     c = math.sqrt(max(0.0, 1.0 - cfg.rho * cfg.rho))
+    def noise(*shape):
+        x = torch.randn(*shape, generator=g, device=dev, dtype=torch.float32)
+        if cfg.noise == "student_t5":     # t_5 = normal / sqrt(chi2_5 / 5), rescaled to unit variance (var of t_5 is 5/3)
+            chi2 = torch.zeros(*shape, device=dev, dtype=torch.float32)
+            for _ in range(5):
+                chi2 += torch.randn(*shape, generator=g, device=dev, dtype=torch.float32) ** 2
+            x = x / torch.sqrt(chi2 / 5.0) * math.sqrt(3.0 / 5.0)
+        return x
+
     for r0 in range(0, rows, row_chunk):
         r1 = min(rows, r0 + row_chunk)
-        gz = torch.randn(r1 - r0, N, generator=g, device=dev, dtype=torch.float32)
-        h = torch.randn(r1 - r0, n, generator=g, device=dev, dtype=torch.float32)
+        gz = noise(r1 - r0, N)
+        h = noise(r1 - r0, n)
         if cfg.drafter_kind == "probs":
             # C5 recipe: the drafter is drawn first, the target copies a correlated part of it.
             y = cfg.sigma * h
