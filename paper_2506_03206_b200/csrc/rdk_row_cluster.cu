@@ -216,7 +216,8 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
     const size_t zb_bytes = ((size_t)Ls * sizeof(TZ) + 127) & ~size_t(127);
     const size_t yb_bytes = ((size_t)(cap + 16) * sizeof(TY) + 127) & ~size_t(127);
     TZ* zbuf = reinterpret_cast<TZ*>(dsm);
-    TY* ybuf[2] = {reinterpret_cast<TY*>(dsm + zb_bytes), reinterpret_cast<TY*>(dsm + zb_bytes + yb_bytes)};
+    // the two drafter buffers, addressed by arithmetic on the shared array (keeps them in the shared address space)
+    auto ybuf_at = [&](int b) -> TY* { return reinterpret_cast<TY*>(dsm + zb_bytes + (b ? yb_bytes : 0)); };
     float* ezb = reinterpret_cast<float*>(dsm + zb_bytes + 2 * yb_bytes);   // e_z of the staged kept tokens
 
     __shared__ __align__(16) float4 segv[CW];
@@ -273,17 +274,17 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
             if (warp == CW - 1) {
                 const YPlan yp = plan_y<TY>(ysrc + r0, kcs);
                 if (lane < len - len8) zbuf[len8 + lane] = zsrc[len8 + lane];
-                if (lane >= 8 && lane < 8 + yp.head) { const int il = lane - 8; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
-                if (lane >= 16 && lane < 16 + yp.tail) { const int il = yp.head + yp.mid + lane - 16; ybuf[b][yp.sh + il] = ysrc[r0 + il]; }
+                if (lane >= 8 && lane < 8 + yp.head) { const int il = lane - 8; ybuf_at(b)[yp.sh + il] = ysrc[r0 + il]; }
+                if (lane >= 16 && lane < 16 + yp.tail) { const int il = yp.head + yp.mid + lane - 16; ybuf_at(b)[yp.sh + il] = ysrc[r0 + il]; }
                 __syncwarp();
                 if (lane == 0) {
                     bulk_load(&zbar, zbuf, zsrc, zbytes);
-                    bulk_load(&ybar[b], ybuf[b] + yp.sh + yp.head, ysrc + r0 + yp.head, (uint32_t)(yp.mid * sizeof(TY)));
+                    bulk_load(&ybar[b], ybuf_at(b) + yp.sh + yp.head, ysrc + r0 + yp.head, (uint32_t)(yp.mid * sizeof(TY)));
                 }
             }
         } else {
             if (tid < len - len8) zbuf[len8 + tid] = zsrc[len8 + tid];
-            for (int il = tid; il < kcs; il += CT) ybuf[b][il] = ysrc[__ldg(P.slot + r0 + il)];
+            for (int il = tid; il < kcs; il += CT) ybuf_at(b)[il] = ysrc[__ldg(P.slot + r0 + il)];
             __syncthreads();
             if (tid == 0) { bulk_load(&zbar, zbuf, zsrc, zbytes); bulk_load(&ybar[b], nullptr, nullptr, 0); }
         }
@@ -318,7 +319,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         const int b = it & 1;
         const TY* yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
         const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
-        const TY* yb = ybuf[b] + y_shift(row);
+        const TY* yb = ybuf_at(b) + y_shift(row);
         if (tid == 0)   // this row's exchange: nseg records of 32 bytes will arrive from the cluster
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&xbar[b])), "r"(xbytes) : "memory");
         mbar_wait(&zbar, (uint32_t)(it & 1), &fail);
