@@ -333,6 +333,7 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         }
         float my_w = -INFINITY;
         if (KIND == RDK_LOGITS) {
+#pragma unroll 4
             for (int il = rw0 + lane; il < rw1s; il += 32) my_w = fmaxf(my_w, to_float<TY>(yb[il]));
             for (int il = rw1s + lane; il < rw1; il += 32)
                 my_w = fmaxf(my_w, to_float<TY>(yrow[identity ? r0 + il : __ldg(P.slot + r0 + il)]));
@@ -357,17 +358,31 @@ rdk_stream_kernel(const RowParams P, const int C, const int Ls, const int cap, c
         }
         // ---- kept tokens of the warp's range: e_z, e_y (cached), their sums -----------------------------
         float K1 = 0.f, K2 = 0.f, Zq = 0.f, th = 0.f;
+        // groups of four per lane: all loads of a group are issued before its arithmetic and stores
 #pragma unroll
-        for (int k = 0; k < kKeptPerLane; ++k) {
-            if (rw0 + 32 * k >= rw1s) break;                      // warp-uniform
-            const int il = rw0 + lane + 32 * k;
-            if (il < rw1s) {
+        for (int g4 = 0; g4 < kKeptPerLane / 4; ++g4) {
+            if (rw0 + 128 * g4 >= rw1s) break;                    // warp-uniform
+            float zz[4], yy[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int k = 4 * g4 + u;
+                const int il = rw0 + lane + 32 * k;
                 const uint32_t jl = (k & 1) ? (idr[k / 2] >> 16) : (idr[k / 2] & 0xffffu);
-                const float ez = ex2(fmaf(to_float<TZ>(zbuf[jl]), kLog2e, zoff_w));
-                const float y = to_float<TY>(yb[il]);
-                const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff_w)) : y;
-                K1 += ez; K2 = fmaf(ez, ez, K2); Zq += ey; th = fmaf(ez, ey, th);
-                ezb[il] = ez;
+                const bool ok = il < rw1s;
+                zz[u] = ok ? to_float<TZ>(zbuf[jl]) : -INFINITY;
+                yy[u] = ok ? to_float<TY>(yb[il]) : (KIND == RDK_LOGITS ? -INFINITY : 0.f);
+            }
+            float ez[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                ez[u] = ex2(fmaf(zz[u], kLog2e, zoff_w));
+                const float ey = KIND == RDK_LOGITS ? ex2(fmaf(yy[u], kLog2e, yoff_w)) : yy[u];
+                K1 += ez[u]; K2 = fmaf(ez[u], ez[u], K2); Zq += ey; th = fmaf(ez[u], ey, th);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int il = rw0 + lane + 32 * (4 * g4 + u);
+                if (il < rw1s) ezb[il] = ez[u];
             }
         }
         for (int il = rw1s + lane; il < rw1; il += 32) {               // kept tokens beyond the staged part
