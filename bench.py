@@ -34,7 +34,7 @@ UNIT = "tokens/s"
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
 NCU_TRAFFIC = {"sources_sha256": "4220264888ced64cc17664ab87f6c1f3e155a1622e74bca435b7ab2df800fab7",
                "bytes_per_launch": 102812160 + 4858624}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
-KERNEL_SOURCES = ("rdk_row_cluster.cu", "rdk_row.cuh", "rdk_common.cuh")
+KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 
 def _kernel_sources_hash() -> str:

@@ -1,9 +1,27 @@
 // Kept-id index: membership bitmask over the target vocabulary, per-word rank counts and the
 // rank -> drafter-index table.  The intersection I = T n D of Sec. 2 is "ids inside [0, N)";
 // everything else is the out-of-vocabulary set F that Token-Level Intersection drops.
+#include <mutex>
+#include <unordered_map>
+
 #include "rdk_common.cuh"
 
 namespace rdk {
+
+static std::mutex g_order_mu;
+static std::unordered_map<const void*, bool>& order_map() {
+    static std::unordered_map<const void*, bool> m;
+    return m;
+}
+void note_index_order(const void* kept_index, bool ascending_valid) {
+    std::lock_guard<std::mutex> lk(g_order_mu);
+    order_map()[kept_index] = ascending_valid;
+}
+int index_order(const void* kept_index) {
+    std::lock_guard<std::mutex> lk(g_order_mu);
+    auto it = order_map().find(kept_index);
+    return it == order_map().end() ? -1 : (it->second ? 1 : 0);
+}
 
 __global__ void idx_clear_kernel(int32_t* header, uint32_t* mask, int32_t* slot, int words, int N, int n) {
     const int g = blockIdx.x * blockDim.x + threadIdx.x;
@@ -126,6 +144,7 @@ extern "C" int rdk_prepare_ids(const int32_t* kept_ids, int32_t n, int32_t N, vo
     RDK_CUDA(cudaMemcpyAsync(host_hdr, header, sizeof(host_hdr), cudaMemcpyDeviceToHost, s));
     RDK_CUDA(cudaStreamSynchronize(s));
     if (n_valid_host) *n_valid_host = host_hdr[kHdrValid];
+    note_index_order(kept_index, host_hdr[kHdrIdentity] != 0 && host_hdr[kHdrValid] == n);
     if (host_hdr[kHdrDup]) {
         set_error("rdk_prepare_ids: two drafter indices map to the same target token");
         return RDK_ERR_BAD_IDS;

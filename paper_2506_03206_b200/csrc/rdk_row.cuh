@@ -23,9 +23,10 @@ struct RowParams {
     int32_t* accepted_len;
     float* rec;            // per-row records in the workspace
     int32_t* counters;     // per (sequence, trial) arrival counters in the workspace
+    unsigned char* xrec;   // per (row, CTA of the group) published partial records in the workspace
 };
 
-constexpr int kRecFloats = 16 + 4 * 128;  // per-row record: 16 scalars + 4 sums for each of up to 128 segments
+constexpr int kRecFloats = 16 + 4 * 256;  // per-row record: 16 scalars + 4 sums for each of up to 256 segments
 
 // running (max, sum) pair of a soft-max denominator; `b` is a second sum on the same scale
 struct MS { float m, s, b; };
@@ -117,7 +118,7 @@ __device__ __forceinline__ int pick_in_segment(const float (&x)[kVec], float rem
 }
 
 
-// Launches the cluster kernel for the linear path when the problem qualifies; returns
+// Launches the streaming kernels for the linear path when the problem qualifies; returns
 // cudaErrorNotSupported (and launches nothing) when the generic kernel has to be used.
 cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s);
 size_t cluster_workspace_bytes(int rows, int batch, int trials);

@@ -1,0 +1,930 @@
+// Two-kernel form of the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8) for N >= 4096
+// and kept ids in ascending order.
+//
+// Kernel 1 (rdk_stream_kernel): a persistent grid of G groups of C CTAs, 16 warps each.  Group g
+// takes rows g, g + G, ...; within a row, warp w of CTA c owns the contiguous token range
+// ("segment") s = 16 c + w.  Every warp runs its own pipeline: a ring of NS shared-memory stages
+// filled by TMA bulk copies (its slice of the target logits and the matching contiguous run of
+// drafter values), so a row is read from HBM exactly once and no block-wide barrier exists.
+//   first visit  A(row): maxima, sum of e = exp(z - max) over the segment, and over the segment's
+//                        kept tokens sum e_z, sum e_y, sum e_z e_y; (e_z, e_y) pairs are cached.
+//   exchange           : the last warp of a CTA to finish A(row) folds the 16 warp records into one
+//                        and publishes it in global memory as five 64-bit words, each a value paired
+//                        with a per-call tag (so every word validates itself and no fence is needed);
+//                        one warp per CTA later polls the C records of the row.
+//   second visit B(row): runs after A(next row), so the exchange latency is hidden; it revisits the
+//                        cached pairs for sum min(p, q~) and writes the segment's sums.
+// Kernel 2 (rdk_draw_kernel): one CTA per (row, trial) turns the record into draws: it locates the
+// segment by prefix sums, re-reads that one segment (usually still in L2), picks the token, runs
+// the rejection test and the residual draw, and counts the accepted prefix of each sequence.
+//
+// Arithmetic, with p = softmax(z), q' = TLI(softmax(y)), x_j = p_j / N <= 2^-12:
+//   w_j = (N q'_j + theta p_j) / (N + p_j) = (q'_j + theta x_j) / (1 + x_j)
+//       = q'_j + x_j (theta - q'_j) + O(x_j^2)          (dropped terms are below 2^-24 of the total)
+// * A token the drafter does not keep has q'_j = 0, hence w_j / S < p_j: its share of
+//   alpha = sum min(p, q~) is w_j / S and its residual is p_j - w_j / S.  Such tokens enter only
+//   through sum p_j per segment, which comes out of the soft-max sweep itself.
+// * S = sum_j w_j = 1 + O(N^-2), because sum q' = 1 and sum q'_j p_j = theta cancel the
+//   first-order terms; it is taken as 1.
+#include <atomic>
+#include <chrono>
+
+#include "rdk_row.cuh"
+
+namespace rdk {
+
+constexpr int kSW = 16;                  // warps (= segments) per CTA of kernel 1
+constexpr int kSThreads = (kSW + 1) * 32;   // the streaming warps and the exchange warp
+constexpr int kMaxGroup = 16;            // CTAs that share a row
+constexpr int kMaxSeg = kMaxGroup * kSW; // 256, matches kRecFloats
+constexpr int kMinStreamN = 4096;
+constexpr unsigned kSpinLimit = 1u << 20;
+constexpr unsigned kSuspendHint = 20000;  // time a waiting thread may stay suspended per try, in ns
+constexpr int kDT = 256;                 // threads per CTA of kernel 2: 4 warps for the draft, 4 for the residual
+constexpr int kGW = kDT / 64;            // warps per group of kernel 2
+constexpr int kMaxChunks = 128;          // 256-token chunks per segment
+constexpr int kXrecBytes = 64;           // one published CTA record: five (value, tag) words, padded
+
+// record layout (floats): 16 scalars, then 4 per segment
+enum { kRecOffg = 0, kRecInvZp, kRecYoffg, kRecInvZq, kRecTheta, kRecInvN, kRecInvS, kRecS };
+
+struct Scal { float offg, inv_zp, yoffg, inv_zq, theta, inv_n, inv_s; };
+
+struct StreamGeo {
+    int C, G;              // CTAs per group, groups
+    int Lw;                // tokens per segment (multiple of 8)
+    int ST;                // tokens the sweep covers per stage: Lw rounded up to 256
+    int NS;                // stages per warp
+    int zstage;            // bytes per target stage: ST * sizeof(TZ) + 16 (the last 16 bytes hold -inf)
+    int ycap;              // kept-token slots per warp that are staged and cached (multiple of 64)
+    int ystage;            // bytes per drafter stage
+    uint32_t tag;          // value that marks a record word as written by this call
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+template <typename T> __device__ __forceinline__ T neg_inf();
+template <> __device__ __forceinline__ float neg_inf<float>() { return -INFINITY; }
+template <> __device__ __forceinline__ __nv_bfloat16 neg_inf<__nv_bfloat16>() { return __float2bfloat16_rn(-INFINITY); }
+template <typename T> __device__ __forceinline__ T zero_of();
+template <> __device__ __forceinline__ float zero_of<float>() { return 0.f; }
+template <> __device__ __forceinline__ __nv_bfloat16 zero_of<__nv_bfloat16>() { return __float2bfloat16_rn(0.f); }
+
+// number of kept ids below token j (j may equal N)
+__device__ __forceinline__ int rank_at(const RowParams& P, int j, int n_valid) {
+    if (j >= P.N) return n_valid;
+    const uint32_t word = __ldg(P.mask + (j >> 5));
+    return __ldg(P.rank + (j >> 5)) + __popc(word & ((1u << (j & 31)) - 1u));
+}
+
+// w_j for given p_j and q'_j:  (q' + theta x) (1 - x + x^2),  x = p / N
+__device__ __forceinline__ float taylor_w(const Scal& c, float p, float qp) {
+    const float x = p * c.inv_n;
+    return fmaf(c.theta, x, qp) * fmaf(x, x - 1.f, 1.f);
+}
+
+__device__ __forceinline__ bool index_matches(const RowParams& P) {
+    return P.header[kHdrMagic] == kIdxMagic && P.header[kHdrN] == P.N && P.header[kHdrn] == P.n;
+}
+
+// ---- packed fp32 pairs ---------------------------------------------------------------------------
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(*reinterpret_cast<unsigned long long*>(&d))
+        : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)),
+          "l"(*reinterpret_cast<unsigned long long*>(&c)));
+    return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    float2 d;
+    asm("add.rn.f32x2 %0, %1, %2;"
+        : "=l"(*reinterpret_cast<unsigned long long*>(&d))
+        : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+    return d;
+}
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
+    float2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;"
+        : "=l"(*reinterpret_cast<unsigned long long*>(&d))
+        : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+    return d;
+}
+__device__ __forceinline__ float2 splat(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float2 ex2_2(float2 x) { return make_float2(ex2(x.x), ex2(x.y)); }
+
+// ---- shared-memory access by 32-bit shared address -----------------------------------------------
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t a) {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, float x, float y, float z, float w) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
+}
+
+// one target logit at shared byte address a, as fp32
+template <typename TZ> __device__ __forceinline__ float lds_z(uint32_t a);
+template <> __device__ __forceinline__ float lds_z<__nv_bfloat16>(uint32_t a) { return __uint_as_float(lds16(a) << 16); }
+template <> __device__ __forceinline__ float lds_z<float>(uint32_t a) { return __uint_as_float(lds32(a)); }
+
+// two consecutive drafter values at shared byte address a (aligned to the pair), as fp32
+template <typename TY> __device__ __forceinline__ float2 lds_ypair(uint32_t a);
+template <> __device__ __forceinline__ float2 lds_ypair<__nv_bfloat16>(uint32_t a) {
+    const uint32_t w = lds32(a);
+    return make_float2(bf16_lo(w), bf16_hi(w));
+}
+template <> __device__ __forceinline__ float2 lds_ypair<float>(uint32_t a) {
+    const uint2 w = lds64(a);
+    return make_float2(__uint_as_float(w.x), __uint_as_float(w.y));
+}
+
+// maximum of the 8 logits (bf16) / 4 logits (fp32) in one 16-byte vector
+template <typename TZ> struct MaxAcc;
+template <> struct MaxAcc<float> {
+    static constexpr int kPer = 4;
+    float m = -INFINITY;
+    __device__ __forceinline__ void push(uint4 q) {
+        m = fmaxf(fmaxf(m, __uint_as_float(q.x)), fmaxf(__uint_as_float(q.y), fmaxf(__uint_as_float(q.z), __uint_as_float(q.w))));
+    }
+    __device__ __forceinline__ float result() const { return m; }
+};
+template <> struct MaxAcc<__nv_bfloat16> {
+    static constexpr int kPer = 8;
+    __nv_bfloat162 m2 = __float2bfloat162_rn(-INFINITY);
+    __device__ __forceinline__ void push(uint4 q) {
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.z));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+    }
+    __device__ __forceinline__ float result() const { return fmaxf(__low2float(m2), __high2float(m2)); }
+};
+
+// sum of e = 2^(z log2e + off) over the logits of one 16-byte vector, two packed accumulators
+template <typename TZ> __device__ __forceinline__ void exp_sum_vec(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb);
+template <> __device__ __forceinline__ void exp_sum_vec<__nv_bfloat16>(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb) {
+    const float2 e0 = ex2_2(ffma2(make_float2(bf16_lo(q.x), bf16_hi(q.x)), scale, off));
+    const float2 e1 = ex2_2(ffma2(make_float2(bf16_lo(q.y), bf16_hi(q.y)), scale, off));
+    const float2 e2 = ex2_2(ffma2(make_float2(bf16_lo(q.z), bf16_hi(q.z)), scale, off));
+    const float2 e3 = ex2_2(ffma2(make_float2(bf16_lo(q.w), bf16_hi(q.w)), scale, off));
+    Ea = fadd2(Ea, e0); Eb = fadd2(Eb, e1); Ea = fadd2(Ea, e2); Eb = fadd2(Eb, e3);
+}
+template <> __device__ __forceinline__ void exp_sum_vec<float>(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb) {
+    const float2 e0 = ex2_2(ffma2(make_float2(__uint_as_float(q.x), __uint_as_float(q.y)), scale, off));
+    const float2 e1 = ex2_2(ffma2(make_float2(__uint_as_float(q.z), __uint_as_float(q.w)), scale, off));
+    Ea = fadd2(Ea, e0); Eb = fadd2(Eb, e1);
+}
+
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* fail) {
+    unsigned spins = 0;
+    uint32_t done = 0;
+    while (!done) {
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar), "r"(parity), "r"(kSuspendHint) : "memory");
+        if (!done && (++spins > kSpinLimit || ((spins & 1023u) == 0 && *reinterpret_cast<volatile int*>(fail)))) {
+            atomicExch(fail, 1);      // give up: the host reads RDK_ERR_TIMEOUT
+            break;
+        }
+    }
+}
+
+// (value, tag) words in global memory: one 64-bit relaxed access each, so a reader sees a value
+// together with the tag that was stored with it
+__device__ __forceinline__ void st_tagged(unsigned char* p, float v, uint32_t tag) {
+    const unsigned long long w = ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(v);
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_tagged(const unsigned char* p) {
+    unsigned long long w;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(w) : "l"(p) : "memory");
+    return w;
+}
+__device__ __forceinline__ int ld_volatile_s32(const int* p) {
+    int v;
+    asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+
+// Combine per-lane partial soft-max records (sum e, sum e_y, sum e e_y on the scales m, my) over
+// the warp; lanes without a record pass m = my = -inf and zeros.
+__device__ __forceinline__ void combine_records(float& E1, float& Zq, float& th, float& m, float& my) {
+    const float mm = warp_max(m), mmy = warp_max(my);
+    const float f = m > -INFINITY ? ex2((m - mm) * kLog2e) : 0.f;
+    const float g = my > -INFINITY ? ex2((my - mmy) * kLog2e) : 0.f;
+    E1 = warp_sum(E1 * f); Zq = warp_sum(Zq * g); th = warp_sum(th * f * g);
+    m = mm; my = mmy;
+}
+
+// ------------------------------------------------------------------------------------------------
+// kernel 1
+// ------------------------------------------------------------------------------------------------
+// Sums of four per-lane values over the warp with 6 shuffles: afterwards lanes 0-7 hold the total of
+// v0, lanes 8-15 of v1, lanes 16-23 of v2, lanes 24-31 of v3.
+__device__ __forceinline__ float warp_sum4(float v0, float v1, float v2, float v3, int lane) {
+    const bool up = lane & 16;
+    float a = up ? v2 : v0, b = up ? v3 : v1;
+    a += __shfl_xor_sync(0xffffffffu, up ? v0 : v2, 16);
+    b += __shfl_xor_sync(0xffffffffu, up ? v1 : v3, 16);
+    const bool odd = lane & 8;
+    float k = odd ? b : a;
+    k += __shfl_xor_sync(0xffffffffu, odd ? a : b, 8);
+    k += __shfl_xor_sync(0xffffffffu, k, 4);
+    k += __shfl_xor_sync(0xffffffffu, k, 2);
+    k += __shfl_xor_sync(0xffffffffu, k, 1);
+    return k;
+}
+__device__ __forceinline__ float warp_max_redux(float v) {
+    float m;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(m) : "f"(v));
+    return m;
+}
+
+// NIT > 0: the sweep over a stage takes exactly NIT 16-byte vectors per lane, kept in registers
+// between the maximum and the exponential pass; NIT = 0: any stage length, two passes over shared memory.
+template <typename TZ, typename TY, int KIND, int NIT>
+__global__ void __launch_bounds__(kSThreads, 1)
+rdk_stream_kernel(const RowParams P, const StreamGeo g) {
+    extern __shared__ __align__(128) unsigned char dsm[];
+    __shared__ __align__(16) float wrec[2][kSW][8];   // [row parity][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), max z, max y
+    __shared__ __align__(16) float scal[2][8];        // [row parity]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta, m, my
+    __shared__ __align__(8) unsigned long long abar[2];   // [row parity]: the 16 warp records of the row are in wrec[]
+    __shared__ __align__(8) unsigned long long rbar[2];   // [row parity]: the row scalars are in scal[]
+    __shared__ int fail;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grp = blockIdx.x / g.C, crank = blockIdx.x % g.C;
+
+    if (!index_matches(P)) {   // same decision in every CTA of the grid; nothing is in flight yet
+        if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
+        return;
+    }
+    const int n_valid = P.header[kHdrValid];
+    if (!P.header[kHdrIdentity] || n_valid != P.n) {   // not the index the host was told about
+        if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
+        return;
+    }
+    // the draw kernel may be scheduled already; it waits for this whole grid before reading the records
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    if (tid == 0) {
+        fail = 0;
+        for (int k = 0; k < 2; ++k) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&abar[k])), "r"(kSW));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&rbar[k])));
+        }
+    }
+    const int rows_g = grp < P.rows ? (P.rows - grp + g.G - 1) / g.G : 0;
+    const float inv_n = 1.f / (float)P.N;
+    constexpr int kZPer = 16 / (int)sizeof(TZ);          // logits per 16 bytes
+
+    // ---- this warp's segment, its kept tokens, its share of shared memory -------------------------
+    const int cw = warp < kSW ? warp : 0;                // the exchange warp owns no segment
+    const int seg = crank * kSW + cw;
+    const long long j0l = (long long)seg * g.Lw;
+    const int j0 = (int)(j0l < P.N ? j0l : P.N);
+    const int len = max(0, min(P.N - j0, g.Lw));
+    const int len_v = len & ~(kZPer - 1);
+    const uint32_t zbytes = (uint32_t)len_v * (uint32_t)sizeof(TZ);
+    const int r_lo = rank_at(P, j0, n_valid), r_hi = rank_at(P, j0 + len, n_valid);
+    const int kc = r_hi - r_lo;
+    const int dummy = r_lo & 1;            // slot 0 of the warp's pair grid belongs to the previous segment
+    const int r0 = r_lo - dummy;           // drafter index of slot 0
+    const int kcp = kc + dummy;            // slots in use
+    const int kcs = min(kcp, g.ycap);      // ... of which staged and cached
+    const int nsteps = (kcs + 63) >> 6;    // steps of 32 lanes x 2 slots
+
+    const size_t off_y = (size_t)kSW * g.NS * g.zstage;
+    const size_t off_cache = off_y + (size_t)kSW * g.NS * g.ystage;
+    const size_t off_goff = off_cache + (size_t)kSW * 2 * g.ycap * 8;
+    const size_t off_bar = off_goff + (size_t)kSW * g.ycap * 2;
+    const uint32_t dsm_a = smem_u32(dsm);
+    const uint32_t zst_a = dsm_a + (uint32_t)(cw * g.NS * g.zstage);
+    const uint32_t yst_a = dsm_a + (uint32_t)(off_y + (size_t)cw * g.NS * g.ystage);
+    const uint32_t cache_a = dsm_a + (uint32_t)(off_cache + (size_t)cw * 2 * g.ycap * 8);
+    const uint32_t goff_a = dsm_a + (uint32_t)(off_goff + (size_t)cw * g.ycap * 2);
+    const uint32_t bar_a = dsm_a + (uint32_t)(off_bar + (size_t)cw * g.NS * 8);
+    unsigned char* zst_p = dsm + (size_t)cw * g.NS * g.zstage;
+    unsigned char* yst_p = dsm + off_y + (size_t)cw * g.NS * g.ystage;
+
+    if (warp < kSW) {
+        if (lane == 0)
+            for (int s = 0; s < g.NS; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a + 8u * s));
+        // beyond the segment (and the 16 spare bytes of every stage): weight 0
+        for (int s = 0; s < g.NS; ++s) {
+            TZ* zs = reinterpret_cast<TZ*>(zst_p + (size_t)s * g.zstage);
+            for (int t = len + lane; t < g.ST + kZPer; t += 32) zs[t] = neg_inf<TZ>();
+        }
+        // shared byte offset (within a stage, 16 bits) of the target logit of every cached slot; unused
+        // slots point at the spare -inf
+        uint32_t* goff_p = reinterpret_cast<uint32_t*>(dsm + off_goff + (size_t)cw * g.ycap * 2);
+        const uint32_t spare = (uint32_t)g.ST * (uint32_t)sizeof(TZ);
+        for (int q = lane; q < nsteps * 32; q += 32) {
+            uint32_t o[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int il = 2 * q + h;
+                o[h] = spare;
+                if (il < kcs && !(dummy && il == 0)) o[h] = (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ);
+            }
+            goff_p[q] = o[0] | (o[1] << 16);
+        }
+    }
+    if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+
+    if (warp == kSW) {
+        // ---- exchange warp: per row, fold the CTA's 16 warp records into one, publish it, collect the
+        // ---- C records of the row and leave the row scalars in shared memory, ahead of the second visits
+        for (int it = 0; it < rows_g; ++it) {
+            const int par = it & 1;
+            const uint32_t ph = (uint32_t)((it >> 1) & 1);
+            const long long row = grp + (long long)it * g.G;
+            mbar_wait(smem_u32(&abar[par]), ph, &fail);
+            float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY;
+            if (lane < kSW) {
+                const volatile float* wr = &wrec[par][lane][0];
+                E1 = wr[0]; Zq = wr[2]; th = wr[3]; m = wr[4]; my = wr[5];
+            }
+            combine_records(E1, Zq, th, m, my);
+            if (lane == 0) {
+                unsigned char* xr = P.xrec + ((size_t)row * g.C + crank) * kXrecBytes;
+                st_tagged(xr, E1, g.tag); st_tagged(xr + 8, Zq, g.tag); st_tagged(xr + 16, th, g.tag);
+                st_tagged(xr + 24, m, g.tag); st_tagged(xr + 32, my, g.tag);
+            }
+            E1 = 0.f; Zq = 0.f; th = 0.f; m = -INFINITY; my = -INFINITY;
+            if (lane < g.C) {
+                const unsigned char* xr = P.xrec + ((size_t)row * g.C + lane) * kXrecBytes;
+                unsigned long long w[5];
+                unsigned spins = 0;
+                for (;;) {
+                    bool ok = true;
+#pragma unroll
+                    for (int k = 0; k < 5; ++k) w[k] = ld_tagged(xr + 8 * k);
+#pragma unroll
+                    for (int k = 0; k < 5; ++k) ok = ok && (uint32_t)(w[k] >> 32) == g.tag;
+                    if (ok) break;
+                    if (++spins > kSpinLimit || ld_volatile_s32(&fail)) { atomicExch(&fail, 1); break; }
+                }
+                E1 = __uint_as_float((uint32_t)w[0]); Zq = __uint_as_float((uint32_t)w[1]); th = __uint_as_float((uint32_t)w[2]);
+                m = __uint_as_float((uint32_t)w[3]); my = __uint_as_float((uint32_t)w[4]);
+            }
+            combine_records(E1, Zq, th, m, my);
+            const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
+            const float theta = th * inv_zp * inv_zq;
+            if (lane == 0) {
+                float* sc = scal[par];
+                sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq;
+                sc[4] = theta; sc[5] = m; sc[6] = my;
+                if (crank == 0) {
+                    float* rec = P.rec + row * kRecFloats;
+                    rec[kRecOffg] = sc[0]; rec[kRecInvZp] = inv_zp; rec[kRecYoffg] = sc[2]; rec[kRecInvZq] = inv_zq;
+                    rec[kRecTheta] = theta; rec[kRecInvN] = inv_n; rec[kRecInvS] = 1.f; rec[kRecS] = 1.f;
+                }
+                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[par])) : "memory");
+            }
+            if (crank == 0 && P.counters && row % P.positions == 0)
+                for (int t = lane; t < P.trials; t += 32) P.counters[(row / P.positions) * P.trials + t] = 0;
+        }
+    } else {
+        // ---- streaming warps ---------------------------------------------------------------------------
+        const long long zstep = (long long)g.G * P.target_stride, ystep = (long long)g.G * P.drafter_stride;
+        const uintptr_t y_end16 = reinterpret_cast<uintptr_t>(static_cast<const TY*>(P.drafter) +
+                                                              (long long)(P.rows - 1) * P.drafter_stride + P.n) & ~uintptr_t(15);
+        // next row to load, and the stage it goes to
+        const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0;
+        const TY* ny = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + r0;
+        int is = 0;
+        // Loads of one row into stage `is`.  Lanes stage the few elements a 16-byte bulk copy cannot
+        // cover with plain stores, then lane 0 arms the barrier and starts the copies.
+        auto issue_next = [&]() {
+            TZ* zs = reinterpret_cast<TZ*>(zst_p + (size_t)is * g.zstage);
+            unsigned char* ys = yst_p + (size_t)is * g.ystage;
+            const uintptr_t b0 = reinterpret_cast<uintptr_t>(ny), b1 = b0 + (uintptr_t)kcs * sizeof(TY);
+            const uintptr_t a0 = b0 & ~uintptr_t(15);
+            uintptr_t a1 = (b1 + 15) & ~uintptr_t(15);
+            if (a1 > y_end16) a1 = y_end16 > a0 ? y_end16 : a0;     // never read past the drafter buffer
+            const uint32_t ybytes = kcs ? (uint32_t)(a1 - a0) : 0u;
+            if (len > len_v) {
+                if (lane < len - len_v) zs[len_v + lane] = nz[len_v + lane];
+            }
+            if (kcs && a1 < b1) {
+                const uintptr_t t0 = a1 > b0 ? a1 : b0;
+                const int nt = (int)((b1 - t0) / sizeof(TY));
+                if (lane < nt) reinterpret_cast<TY*>(ys + (t0 - a0))[lane] = reinterpret_cast<const TY*>(t0)[lane];
+            }
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t bar = bar_a + 8u * is;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                if (zbytes + ybytes == 0) {
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+                } else {
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(zbytes + ybytes) : "memory");
+                    if (zbytes)
+                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                     ::"r"(zst_a + (uint32_t)(is * g.zstage)), "l"(nz), "r"(zbytes), "r"(bar) : "memory");
+                    if (ybytes)
+                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                     ::"r"(yst_a + (uint32_t)(is * g.ystage)), "l"(a0), "r"(ybytes), "r"(bar) : "memory");
+                }
+            }
+            nz += zstep; ny += ystep;
+            is = is + 1 == g.NS ? 0 : is + 1;
+        };
+        for (int itx = 0; itx < g.NS && itx < rows_g; ++itx) issue_next();
+
+        const float2 l2e = splat(kLog2e);
+
+        // ---- second visit of local row `itb` -----------------------------------------------------
+        auto second_visit = [&](int itb) {
+            const int par = itb & 1;
+            const long long row = grp + (long long)itb * g.G;
+            mbar_wait(smem_u32(&rbar[par]), (uint32_t)((itb >> 1) & 1), &fail);
+            const float4 s0 = *reinterpret_cast<const float4*>(&scal[par][0]);   // -m log2e, 1/Zp, -my log2e, 1/Zq
+            const float4 s1 = *reinterpret_cast<const float4*>(&scal[par][4]);   // theta, m, my
+            const float4 w0 = *reinterpret_cast<const float4*>(&wrec[par][warp][0]);   // this warp's sums of the row
+            const float2 w1 = *reinterpret_cast<const float2*>(&wrec[par][warp][4]);   // ... and maxima
+            const float theta = s1.x;
+            const float fz = (w1.x > -INFINITY ? ex2((w1.x - s1.y) * kLog2e) : 0.f) * s0.y;
+            const float fy = (KIND == RDK_LOGITS ? (w1.y > -INFINITY ? ex2((w1.y - s1.z) * kLog2e) : 0.f) : 1.f) * s0.w;
+            // kept tokens: sum of min(p, q~), q~ = q' + x (theta - q'), from the cached (e_z, e_y)
+            const float2 fz2 = splat(fz), fy2 = splat(fy), xs2 = splat(fz * inv_n), th2 = splat(theta), neg1 = splat(-1.f);
+            float2 ak2 = splat(0.f);
+            const uint32_t cb = cache_a + (uint32_t)(par * g.ycap * 8) + (uint32_t)lane * 16u;
+#pragma unroll 4
+            for (int st = 0; st < nsteps; ++st) {
+                const uint4 c4 = lds128(cb + (uint32_t)st * 512u);
+                const float2 ez = make_float2(__uint_as_float(c4.x), __uint_as_float(c4.y));
+                const float2 ey = make_float2(__uint_as_float(c4.z), __uint_as_float(c4.w));
+                const float2 p = fmul2(ez, fz2), qp = fmul2(ey, fy2), x = fmul2(ez, xs2);
+                const float2 w = ffma2(x, ffma2(qp, neg1, th2), qp);
+                ak2 = fadd2(ak2, make_float2(fminf(p.x, w.x), fminf(p.y, w.y)));
+            }
+            float ak = ak2.x + ak2.y;
+            if (kcp > kcs) {   // kept tokens beyond the cache: from global memory again
+                const TZ* zrow = static_cast<const TZ*>(P.target) + row * P.target_stride;
+                const TY* yrow = static_cast<const TY*>(P.drafter) + row * P.drafter_stride;
+                const float zoff = w1.x > -INFINITY ? -w1.x * kLog2e : 0.f, yoff = w1.y > -INFINITY ? -w1.y * kLog2e : 0.f;
+                for (int il = kcs + lane; il < kcp; il += 32) {
+                    const float ez = ex2(fmaf(to_float<TZ>(zrow[__ldg(P.ids + r0 + il)]), kLog2e, zoff));
+                    const float y = to_float<TY>(yrow[r0 + il]);
+                    const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
+                    const float p = ez * fz, qp = ey * fy;
+                    ak += fminf(p, fmaf(p * inv_n, theta - qp, qp));
+                }
+            }
+            ak = warp_sum(ak);
+            if (lane == 0) {
+                // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
+                const float segP = w0.x * fz;
+                const float oov = theta * inv_n * fmaxf(0.f, w0.x - w0.y) * fz;
+                const float xs = fz * inv_n;
+                const float Kw = fy * w0.z - fy * xs * w0.w + theta * xs * w0.y;
+                const float a_s = oov + ak;
+                reinterpret_cast<float4*>(P.rec + row * kRecFloats + 16)[seg] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP - a_s), segP);
+            }
+        };
+
+        // ---- main loop: first visit of row it, reload of its stage, second visit of row it - 1 ----
+        const TY* cy = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + r0;   // slot 0 of the current row
+        int s = 0;
+        uint32_t sph = 0;
+        for (int it = 0; it < rows_g; ++it) {
+            const int par = it & 1;
+            const uint32_t zs_a = zst_a + (uint32_t)(s * g.zstage);
+            const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(cy) & 15u);      // slot 0 sits this many bytes into the stage
+            const uint32_t ys_a = yst_a + (uint32_t)(s * g.ystage) + shb;
+            mbar_wait(bar_a + 8u * s, sph, &fail);
+
+            // slots of the pair grid that hold no kept token of this segment read as weight 0
+            {
+                TY* yp = reinterpret_cast<TY*>(yst_p + (size_t)s * g.ystage + shb);
+                const TY fill = KIND == RDK_LOGITS ? neg_inf<TY>() : zero_of<TY>();
+                if (dummy && lane == 0 && kcs > 0) yp[0] = fill;
+                for (int il = kcs + lane; il < nsteps * 64; il += 32) yp[il] = fill;
+                __syncwarp();
+            }
+
+            // maxima of the segment and of its kept drafter values
+            uint4 zv[NIT > 0 ? NIT : 1];
+            MaxAcc<TZ> mz;
+            if (NIT > 0) {
+#pragma unroll
+                for (int k = 0; k < NIT; ++k) zv[k] = lds128(zs_a + (uint32_t)(k * 32 + lane) * 16u);
+#pragma unroll
+                for (int k = 0; k < NIT; ++k) mz.push(zv[k]);
+            } else {
+#pragma unroll 4
+                for (int t = lane * kZPer; t < g.ST; t += 32 * kZPer) mz.push(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)));
+            }
+            float my_w = KIND == RDK_LOGITS ? -INFINITY : 0.f;
+            if (KIND == RDK_LOGITS) {
+#pragma unroll 4
+                for (int st = 0; st < nsteps; ++st) {
+                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)(st * 64 + lane * 2) * (uint32_t)sizeof(TY));
+                    my_w = fmaxf(my_w, fmaxf(y.x, y.y));
+                }
+                for (int il = kcs + lane; il < kcp; il += 32) my_w = fmaxf(my_w, to_float<TY>(cy[il]));
+                my_w = warp_max_redux(my_w);
+            }
+            const float m_w = warp_max_redux(mz.result());
+            const float zoff = m_w > -INFINITY ? -m_w * kLog2e : 0.f;
+            const float yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
+
+            // soft-max sweep: sum of e over the segment
+            float2 Ea = splat(0.f), Eb = splat(0.f);
+            {
+                const float2 of = splat(zoff);
+                if (NIT > 0) {
+#pragma unroll
+                    for (int k = 0; k < NIT; ++k) exp_sum_vec<TZ>(zv[k], l2e, of, Ea, Eb);
+                } else {
+#pragma unroll 4
+                    for (int t = lane * kZPer; t < g.ST; t += 32 * kZPer)
+                        exp_sum_vec<TZ>(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)), l2e, of, Ea, Eb);
+                }
+            }
+            // kept tokens: e_z, e_y, their sums; the pairs go to the cache
+            float2 K1 = splat(0.f), Zq = splat(0.f), th = splat(0.f);
+            {
+                const float2 zof = splat(zoff), yof = splat(yoff);
+                const uint32_t cb = cache_a + (uint32_t)(par * g.ycap * 8) + (uint32_t)lane * 16u;
+#pragma unroll 2
+                for (int st = 0; st < nsteps; ++st) {
+                    const uint32_t go = lds32(goff_a + (uint32_t)(st * 32 + lane) * 4u);
+                    const float2 z = make_float2(lds_z<TZ>(zs_a + (go & 0xffffu)), lds_z<TZ>(zs_a + (go >> 16)));
+                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)(st * 64 + lane * 2) * (uint32_t)sizeof(TY));
+                    const float2 ez = ex2_2(ffma2(z, l2e, zof));
+                    const float2 ey = KIND == RDK_LOGITS ? ex2_2(ffma2(y, l2e, yof)) : y;
+                    K1 = fadd2(K1, ez); Zq = fadd2(Zq, ey); th = ffma2(ez, ey, th);
+                    sts128(cb + (uint32_t)st * 512u, ez.x, ez.y, ey.x, ey.y);
+                }
+            }
+            float E1s = (Ea.x + Ea.y) + (Eb.x + Eb.y), K1s = K1.x + K1.y, Zqs = Zq.x + Zq.y, ths = th.x + th.y;
+            for (int il = kcs + lane; il < kcp; il += 32) {               // kept tokens beyond the cache
+                const float ez = ex2(fmaf(lds_z<TZ>(zs_a + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ)), kLog2e, zoff));
+                const float y = to_float<TY>(cy[il]);
+                const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
+                K1s += ez; Zqs += ey; ths = fmaf(ez, ey, ths);
+            }
+            const float tot = warp_sum4(E1s, K1s, Zqs, ths, lane);      // lanes 0, 8, 16, 24 hold the four totals
+
+            // the stage is free: bring in the row NS ahead
+            __syncwarp();
+            if (it + g.NS < rows_g) issue_next();
+
+            // hand the warp's record to the exchange warp
+            if ((lane & 7) == 0) wrec[par][warp][lane >> 3] = tot;
+            if (lane == 0) { wrec[par][warp][4] = m_w; wrec[par][warp][5] = my_w; }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&abar[par])) : "memory");
+
+            if (it > 0) second_visit(it - 1);
+            cy += ystep;
+            if (++s == g.NS) { s = 0; sph ^= 1u; }
+        }
+        if (rows_g > 0) second_visit(rows_g - 1);
+    }
+    __syncthreads();
+    if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
+// kernel 2
+// ------------------------------------------------------------------------------------------------
+struct DrawCtx {
+    const void* zrow; const void* yrow; bool zvec;
+    const uint32_t* mask; const int32_t* rank;
+    int N;
+    Scal c;
+};
+
+// p and w of the 8 tokens starting at global token jb (a multiple of 8)
+template <typename TZ, typename TY, int KIND>
+__device__ __forceinline__ void draw_pw(const DrawCtx& d, int jb, float (&p)[kVec], float (&w)[kVec]) {
+    float z[kVec];
+    load8<TZ>(static_cast<const TZ*>(d.zrow), jb, d.N, d.zvec, -INFINITY, z);
+    const uint32_t word = __ldg(d.mask + (jb >> 5));
+    const int rbase = __ldg(d.rank + (jb >> 5));          // issued together with the mask and the logits
+    const int sh = jb & 31;
+    const uint32_t mb = (word >> sh) & 0xffu;
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) {
+        p[k] = ex2(fmaf(z[k], kLog2e, d.c.offg)) * d.c.inv_zp;
+        w[k] = taylor_w(d.c, p[k], 0.f);
+    }
+    if (!mb) return;
+    int r = rbase + __popc(word & ((1u << sh) - 1u));
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) {
+        if (mb & (1u << k)) {
+            const float y = to_float<TY>(static_cast<const TY*>(d.yrow)[r]);     // ascending kept ids: rank = drafter index
+            ++r;
+            const float qp = (KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, d.c.yoffg)) : y) * d.c.inv_zq;
+            w[k] = taylor_w(d.c, p[k], qp);
+        }
+    }
+}
+
+enum { kPickW = 0, kPickR = 1, kPickP = 2 };
+
+template <typename TZ, typename TY, int KIND>
+__device__ __forceinline__ void draw_x(const DrawCtx& d, int what, int jb, int seg_end, float (&p)[kVec], float (&w)[kVec], float (&x)[kVec]) {
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) { p[k] = 0.f; w[k] = 0.f; x[k] = 0.f; }
+    if (jb >= seg_end) return;
+    draw_pw<TZ, TY, KIND>(d, jb, p, w);
+#pragma unroll
+    for (int k = 0; k < kVec; ++k)
+        x[k] = what == kPickW ? w[k] : (what == kPickR ? fmaxf(0.f, p[k] - w[k] * d.c.inv_s) : p[k]);
+}
+
+template <typename TZ, typename TY, int KIND>
+__global__ void __launch_bounds__(kDT)
+rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
+    __shared__ double cdfW[kMaxSeg], cdfR[kMaxSeg], cdfP[kMaxSeg];
+    __shared__ float sums[2][kMaxChunks];
+    __shared__ float alpha_s;
+    __shared__ int res_tok[2];
+    __shared__ float res_p[2], res_w[2];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row = blockIdx.x / P.trials, t = blockIdx.x % P.trials;
+    const float* rec = P.rec + (long long)row * kRecFloats;
+    DrawCtx d;
+    const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
+    const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
+    if (!index_matches(P)) return;                 // kernel 1 has reported it
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // kernel 1 (launched just before) is complete and visible
+    d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
+    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
+    d.c.inv_s = __ldcg(rec + kRecInvS);
+
+    if (warp == 0) {   // prefix sums over the segments, fp64
+        double cw = 0.0, cr = 0.0, cp = 0.0;
+        float alpha_l = 0.f;
+        for (int base = 0; base < nseg; base += 32) {
+            const int s = base + lane;
+            double iw = 0.0, ir = 0.0, ip = 0.0;
+            if (s < nseg) {
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(rec + 16) + s);
+                iw = (double)v.x; alpha_l += v.y; ir = (double)v.z; ip = (double)v.w;
+            }
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double a = __shfl_up_sync(0xffffffffu, iw, o);
+                const double b = __shfl_up_sync(0xffffffffu, ir, o);
+                const double e = __shfl_up_sync(0xffffffffu, ip, o);
+                if (lane >= o) { iw += a; ir += b; ip += e; }
+            }
+            iw += cw; ir += cr; ip += cp;
+            cw = __shfl_sync(0xffffffffu, iw, 31);
+            cr = __shfl_sync(0xffffffffu, ir, 31);
+            cp = __shfl_sync(0xffffffffu, ip, 31);
+            if (s < nseg) { cdfW[s] = iw; cdfR[s] = ir; cdfP[s] = ip; }
+        }
+        alpha_l = warp_sum(alpha_l);
+        if (lane == 0) alpha_s = alpha_l;
+    }
+    __syncthreads();
+    const double S_d = cdfW[nseg - 1], R_d = cdfR[nseg - 1], Pt_d = cdfP[nseg - 1];
+    if (t == 0 && tid == 0) {
+        if (P.alpha) P.alpha[row] = alpha_s;
+        if (P.theta) P.theta[row] = d.c.theta;
+        if (P.S) P.S[row] = (float)S_d;
+        if (P.residual_mass) P.residual_mass[row] = (float)R_d;
+    }
+    const TZ* zrow = static_cast<const TZ*>(P.target) + (long long)row * P.target_stride;
+    d.zrow = zrow; d.yrow = static_cast<const TY*>(P.drafter) + (long long)row * P.drafter_stride;
+    d.zvec = (reinterpret_cast<uintptr_t>(zrow) & 15u) == 0;
+    d.mask = P.mask; d.rank = P.rank; d.N = P.N;
+
+    // group 0 (first half of the warps): the draft draw from w; group 1: the residual draw, computed
+    // alongside (it is only used if the draft is rejected)
+    const int g = warp / kGW, wg = warp % kGW;
+    const bool from_p = !(R_d > 0.0);                 // p and q~ coincide: the replacement comes from p itself
+    const double* cdf = g == 0 ? cdfW : (from_p ? cdfP : cdfR);
+    const int what = g == 0 ? kPickW : (from_p ? kPickP : kPickR);
+    const double thr = g == 0 ? (double)u0 * S_d : (double)u2 * (from_p ? Pt_d : R_d);
+    const int seg = min(first_above(cdf, nseg, thr), nseg - 1);
+    const float rem = (float)(thr - (seg ? cdf[seg - 1] : 0.0));
+    const int seg_lo = (int)min((long long)seg * Lw, (long long)P.N);
+    const int seg_end = (int)min((long long)P.N, (long long)seg_lo + Lw);
+    const int nch = (Lw + kSeg - 1) / kSeg;
+    for (int ch = wg; ch < nch; ch += kGW) {
+        float p[kVec], w[kVec], x[kVec];
+        draw_x<TZ, TY, KIND>(d, what, seg_lo + ch * kSeg + lane * kVec, seg_end, p, w, x);
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < kVec; ++k) s += x[k];
+        s = warp_sum(s);
+        if (lane == 0) sums[g][ch] = s;
+    }
+    __syncthreads();
+    {   // every warp finds the chunk of its group; the warp that owns it picks the token
+        float cum = 0.f, before = 0.f;
+        int chosen = -1, last_pos = -1;
+        for (int ch = 0; ch < nch; ++ch) {
+            const float s = sums[g][ch];
+            if (s > 0.f) {
+                if (chosen < 0 && cum + s > rem) { chosen = ch; before = cum; }
+                last_pos = ch;
+                cum += s;
+            }
+        }
+        float r_in = rem - before;
+        if (chosen < 0) { chosen = last_pos; r_in = INFINITY; }      // rounding: the last positive token
+        if (chosen < 0) {
+            if (wg == 0 && lane == 0) { res_tok[g] = seg_lo; res_p[g] = 0.f; res_w[g] = 0.f; }
+        } else if (chosen % kGW == wg) {
+            float p[kVec], w[kVec], x[kVec];
+            draw_x<TZ, TY, KIND>(d, what, seg_lo + chosen * kSeg + lane * kVec, seg_end, p, w, x);
+            int sel = pick_in_segment(x, r_in, lane);
+            if (sel < 0) sel = 0;
+            float ps = 0.f, ws = 0.f;
+#pragma unroll
+            for (int k = 0; k < kVec; ++k) if (k == (sel & (kVec - 1))) { ps = p[k]; ws = w[k]; }
+            ps = __shfl_sync(0xffffffffu, ps, sel / kVec);
+            ws = __shfl_sync(0xffffffffu, ws, sel / kVec);
+            if (lane == 0) { res_tok[g] = seg_lo + chosen * kSeg + sel; res_p[g] = ps; res_w[g] = ws; }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const int dtok = res_tok[0];
+        const float pd = res_p[0], qd = res_w[0] * d.c.inv_s;
+        const float a_prob = (pd >= qd) ? 1.f : pd / qd;
+        const bool acc = u1 * qd < pd;
+        const long long o = (long long)row * P.trials + t;
+        if (P.draft_token) P.draft_token[o] = dtok;
+        if (P.accepted) P.accepted[o] = acc ? 1 : 0;
+        if (P.accept_prob) P.accept_prob[o] = a_prob;
+        if (P.out_token) P.out_token[o] = acc ? dtok : res_tok[1];
+        if (P.accepted_len && P.accepted && P.counters) {
+            // the last position of a sequence to finish counts the accepted prefix (Algorithm 4 step 7)
+            const int b = row / P.positions;
+            __threadfence();
+            const int old = atomicAdd(P.counters + b * P.trials + t, 1);
+            if (old == P.positions - 1) {
+                __threadfence();
+                int k = 0;
+                const volatile uint8_t* af = P.accepted;
+                while (k < P.positions && af[((long long)b * P.positions + k) * P.trials + t]) ++k;
+                P.accepted_len[b * P.trials + t] = k;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+static size_t stream_smem(const StreamGeo& g) {
+    return (size_t)kSW * ((size_t)g.NS * (g.zstage + g.ystage + 8) + (size_t)g.ycap * 18);   // + cache (2 x 8 bytes) and offsets (2 bytes) per slot
+}
+
+// Group size, segment length, stage count and cache capacity for a vocabulary of N tokens with n
+// kept ids; false when the shapes do not fit shared memory.
+static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
+    const size_t budget = 225 * 1024;      // dynamic shared memory a CTA may ask for, less the static part
+    int C = (N + kSW * 1024 - 1) / (kSW * 1024);
+    if (C > kMaxGroup) C = kMaxGroup;
+    const int per = (N + C * kSW - 1) / (C * kSW);
+    g.C = C;
+    g.Lw = (per + 7) & ~7;
+    g.ST = (g.Lw + 255) & ~255;
+    g.zstage = g.ST * (int)es + 16;
+    if ((g.Lw + kSeg - 1) / kSeg > kMaxChunks || g.zstage > 65535) return false;   // stage offsets are 16-bit
+    const long long expect = ((long long)n * g.Lw + N - 1) / N;
+    long long cap = expect + expect / 8 + 32;
+    const long long most = (long long)(n < g.Lw ? n : g.Lw) + 1;
+    if (cap > most) cap = most;
+    cap = (cap + 63) / 64 * 64;
+    for (g.NS = 3; g.NS >= 2; --g.NS) {
+        long long c = cap;
+        while (c >= 64) {
+            g.ycap = (int)c;
+            g.ystage = (int)((((size_t)c + 16) * ys + 15) & ~size_t(15));
+            if (stream_smem(g) <= budget) return true;
+            if (g.NS > 2) break;          // first give up a stage, then cache capacity
+            c -= 64;
+        }
+    }
+    return false;
+}
+
+template <typename TZ, typename TY, int KIND, int NIT>
+static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s) {
+    auto kern = rdk_stream_kernel<TZ, TY, KIND, NIT>;
+    const size_t smem = stream_smem(g);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    // how many CTAs are resident at once (cached per kernel instance, shared-memory size and device)
+    static thread_local int c_dev = -1, c_ctas = 0;
+    static thread_local size_t c_smem = 0;
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev != c_dev || smem != c_smem) {
+        int sms = 0, per_sm = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kSThreads, smem);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) return cudaErrorNotSupported;
+        c_dev = dev; c_smem = smem; c_ctas = sms * per_sm;
+    }
+    if (c_ctas < g.C) return cudaErrorNotSupported;
+    g.G = c_ctas / g.C;
+    if (g.G > P.rows) g.G = P.rows;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(g.G * g.C), 1, 1);
+    cfg.blockDim = dim3(kSThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;      // the CTAs of a group wait for one another: all must be resident
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kern, P, g);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t dcfg = {};
+    dcfg.gridDim = dim3((unsigned)(P.rows * P.trials), 1, 1);
+    dcfg.blockDim = dim3(kDT, 1, 1);
+    dcfg.dynamicSmemBytes = 0;
+    dcfg.stream = s;
+    cudaLaunchAttribute dattr[1];
+    dattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while kernel 1 drains
+    dattr[0].val.programmaticStreamSerializationAllowed = 1;
+    dcfg.attrs = dattr;
+    dcfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&dcfg, rdk_draw_kernel<TZ, TY, KIND>, P, g.C * kSW, g.Lw);
+}
+
+template <typename TZ, typename TY, int KIND>
+static cudaError_t launch_nit(const RowParams& P, const StreamGeo& g, cudaStream_t s) {
+    // the common stage length (four 16-byte vectors per lane) gets the register-resident sweep
+    if (g.ST == 4 * 32 * (16 / (int)sizeof(TZ))) return launch_stream<TZ, TY, KIND, 4>(P, g, s);
+    return launch_stream<TZ, TY, KIND, 0>(P, g, s);
+}
+
+template <typename TZ, typename TY>
+static cudaError_t launch_kind_s(const RowParams& P, int kind, const StreamGeo& g, cudaStream_t s) {
+    return kind == RDK_LOGITS ? launch_nit<TZ, TY, RDK_LOGITS>(P, g, s) : launch_nit<TZ, TY, RDK_PROBS>(P, g, s);
+}
+
+static size_t ws_off_counters(int rows) { return idx_align((size_t)rows * kRecFloats * sizeof(float)); }
+static size_t ws_off_xrec(int rows, int batch, int trials) { return ws_off_counters(rows) + idx_align((size_t)batch * trials * sizeof(int32_t)); }
+
+size_t cluster_workspace_bytes(int rows, int batch, int trials) {
+    return ws_off_xrec(rows, batch, trials) + idx_align((size_t)rows * kMaxGroup * kXrecBytes);
+}
+
+// A non-zero 32-bit value that differs from the one of every recent call of this process and that
+// stale memory is unlikely to hold.
+static uint32_t next_tag() {
+    static std::atomic<uint32_t> ctr{
+        (uint32_t)std::chrono::high_resolution_clock::now().time_since_epoch().count() * 0x9E3779B9u + 1u};
+    const uint32_t t = ctr.fetch_add(0x9E3779B9u) + 0x9E3779B9u;
+    return t ? t : 0x9E3779B9u;
+}
+
+cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s) {
+    const size_t es = tz == RDK_F32 ? 4 : 2, ys = ty == RDK_F32 ? 4 : 2;
+    if (P.N < kMinStreamN || P.qtilde || P.rows <= 0 || P.trials <= 0 || !ws) return cudaErrorNotSupported;
+    // rows of the target start on 16-byte boundaries; drafter values are read in aligned pairs
+    if ((reinterpret_cast<uintptr_t>(P.target) & 15u) || ((P.target_stride * (long long)es) & 15)) return cudaErrorNotSupported;
+    if ((reinterpret_cast<uintptr_t>(P.drafter) & 15u) || (P.drafter_stride & 1)) return cudaErrorNotSupported;
+    if ((long long)P.rows * P.trials > 0x7fffffffLL) return cudaErrorNotSupported;
+    if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < cluster_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
+    // ascending, valid kept ids only, as recorded when the index was built (kernel 1 re-checks the header)
+    if (index_order(P.header) != 1) return cudaErrorNotSupported;
+    StreamGeo g;
+    if (!plan_stream(P.N, P.n, es, ys, g)) return cudaErrorNotSupported;
+    g.G = 0;
+    g.tag = next_tag();
+    P.rec = static_cast<float*>(ws);
+    P.counters = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + ws_off_counters(P.rows));
+    P.xrec = reinterpret_cast<unsigned char*>(ws) + ws_off_xrec(P.rows, batch, P.trials);
+    if (tz == RDK_F32) return ty == RDK_F32 ? launch_kind_s<float, float>(P, kind, g, s) : launch_kind_s<float, __nv_bfloat16>(P, kind, g, s);
+    return ty == RDK_F32 ? launch_kind_s<__nv_bfloat16, float>(P, kind, g, s) : launch_kind_s<__nv_bfloat16, __nv_bfloat16>(P, kind, g, s);
+}
+
+}  // namespace rdk
