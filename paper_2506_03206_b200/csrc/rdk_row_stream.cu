@@ -34,7 +34,7 @@
 namespace rdk {
 
 constexpr int kSW = 16;                  // warps (= segments) per CTA of kernel 1
-constexpr int kSThreads = (kSW + 1) * 32;   // the streaming warps and the exchange warp
+constexpr int kSThreads = (kSW + 2) * 32;   // the streaming warps, the exchange warp and the load warp
 constexpr int kMaxGroup = 16;            // CTAs that share a row
 constexpr int kMaxSeg = kMaxGroup * kSW; // 256, matches kRecFloats
 constexpr int kMinStreamN = 4096;
@@ -52,12 +52,11 @@ struct Scal { float offg, inv_zp, yoffg, inv_zq, theta, inv_n, inv_s; };
 
 struct StreamGeo {
     int C, G;              // CTAs per group, groups
-    int Lw;                // tokens per segment (multiple of 8)
-    int ST;                // tokens the sweep covers per stage: Lw rounded up to 256
-    int NS;                // stages per warp
-    int zstage;            // bytes per target stage: ST * sizeof(TZ) + 16 (the last 16 bytes hold -inf)
+    int Lw;                // tokens per segment: nv vectors of 16 bytes per lane
+    int nv;
+    int NS;                // stages
     int ycap;              // kept-token slots per warp that are staged and cached (multiple of 64)
-    int ystage;            // bytes per drafter stage
+    int ystage;            // bytes of a warp's drafter region in a stage
     uint32_t tag;          // value that marks a record word as written by this call
 };
 
@@ -223,11 +222,14 @@ __device__ __forceinline__ int ld_volatile_s32(const int* p) {
 
 // Combine per-lane partial soft-max records (sum e, sum e_y, sum e e_y on the scales m, my) over
 // the warp; lanes without a record pass m = my = -inf and zeros.
-__device__ __forceinline__ void combine_records(float& E1, float& Zq, float& th, float& m, float& my) {
-    const float mm = warp_max(m), mmy = warp_max(my);
+__device__ __forceinline__ float warp_sum4(float v0, float v1, float v2, float v3, int lane);
+__device__ __forceinline__ float warp_max_redux(float v);
+__device__ __forceinline__ void combine_records(float& E1, float& Zq, float& th, float& m, float& my, int lane) {
+    const float mm = warp_max_redux(m), mmy = warp_max_redux(my);
     const float f = m > -INFINITY ? ex2((m - mm) * kLog2e) : 0.f;
     const float g = my > -INFINITY ? ex2((my - mmy) * kLog2e) : 0.f;
-    E1 = warp_sum(E1 * f); Zq = warp_sum(Zq * g); th = warp_sum(th * f * g);
+    const float tot = warp_sum4(E1 * f, Zq * g, th * f * g, 0.f, lane);
+    E1 = __shfl_sync(0xffffffffu, tot, 0); Zq = __shfl_sync(0xffffffffu, tot, 8); th = __shfl_sync(0xffffffffu, tot, 16);
     m = mm; my = mmy;
 }
 
@@ -255,16 +257,39 @@ __device__ __forceinline__ float warp_max_redux(float v) {
     return m;
 }
 
-// NIT > 0: the sweep over a stage takes exactly NIT 16-byte vectors per lane, kept in registers
-// between the maximum and the exponential pass; NIT = 0: any stage length, two passes over shared memory.
+// One warp's segment of the vocabulary and the kept tokens inside it.
+struct SegInfo {
+    int j0, len;        // first token, tokens inside [0, N)
+    int r0;             // drafter index of slot 0 of the warp's pair grid (even)
+    int dummy;          // 1 when slot 0 belongs to the previous segment
+    int kcp, kcs;       // slots in use; slots staged and cached
+};
+__device__ __forceinline__ SegInfo seg_info(const RowParams& P, const StreamGeo& g, int seg, int n_valid) {
+    SegInfo si;
+    const long long j0l = (long long)seg * g.Lw;
+    si.j0 = (int)(j0l < P.N ? j0l : P.N);
+    si.len = max(0, min(P.N - si.j0, g.Lw));
+    const int r_lo = rank_at(P, si.j0, n_valid), r_hi = rank_at(P, si.j0 + si.len, n_valid);
+    si.dummy = r_lo & 1;
+    si.r0 = r_lo - si.dummy;
+    si.kcp = r_hi - si.r0;
+    si.kcs = min(si.kcp, g.ycap);
+    return si;
+}
+
+// NIT > 0: a segment is exactly NIT 16-byte vectors per lane, kept in registers between the maximum
+// and the exponential pass; NIT = 0: any segment length, two passes over shared memory.
 template <typename TZ, typename TY, int KIND, int NIT>
 __global__ void __launch_bounds__(kSThreads, 1)
 rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     extern __shared__ __align__(128) unsigned char dsm[];
     __shared__ __align__(16) float wrec[2][kSW][8];   // [row parity][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), max z, max y
-    __shared__ __align__(16) float scal[2][8];        // [row parity]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta, m, my
+    __shared__ __align__(16) float scal[2][8];        // [row parity]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta
+    __shared__ __align__(8) float2 fzy[2][kSW];       // [row parity][warp]: factors that turn the warp's cached e_z, e_y into p, q'
+    __shared__ float akv[2][kSW];                     // [row parity][warp]: sum of min(p, q~) over the warp's kept tokens
     __shared__ __align__(8) unsigned long long abar[2];   // [row parity]: the 16 warp records of the row are in wrec[]
-    __shared__ __align__(8) unsigned long long rbar[2];   // [row parity]: the row scalars are in scal[]
+    __shared__ __align__(8) unsigned long long rbar[2];   // [row parity]: scal[] and fzy[] of the row are set
+    __shared__ __align__(8) unsigned long long bbar[2];   // [row parity]: akv[] of the row is set
     __shared__ int fail;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -282,91 +307,275 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     // the draw kernel may be scheduled already; it waits for this whole grid before reading the records
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+    constexpr int kZPer = 16 / (int)sizeof(TZ);          // logits per 16 bytes
+    const int rows_g = grp < P.rows ? (P.rows - grp + g.G - 1) / g.G : 0;
+    const float inv_n = 1.f / (float)P.N;
+
+    // shared memory: NS stages of [the CTA's slice of a target row | 16 bytes of -inf | one drafter
+    // region per warp], then per warp the (e_z, e_y) cache (two rows) and the gather offsets, then barriers
+    const uint32_t zslice = (uint32_t)kSW * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
+    const uint32_t stage = zslice + 16u + (uint32_t)kSW * (uint32_t)g.ystage;
+    const uint32_t off_cache = (uint32_t)g.NS * stage;
+    const uint32_t off_goff = off_cache + (uint32_t)kSW * 2u * (uint32_t)g.ycap * 8u;
+    const uint32_t off_bar = off_goff + (uint32_t)kSW * (uint32_t)g.ycap * 2u;
+    const uint32_t dsm_a = smem_u32(dsm);
+    const uint32_t full_a = dsm_a + off_bar, empty_a = full_a + 8u * (uint32_t)g.NS;
+
     if (tid == 0) {
         fail = 0;
         for (int k = 0; k < 2; ++k) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&abar[k])), "r"(kSW));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&rbar[k])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bbar[k])), "r"(kSW));
+        }
+        for (int k = 0; k < g.NS; ++k) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_a + 8u * k));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_a + 8u * k), "r"(kSW));
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // beyond the vocabulary, and the 16 spare bytes of every stage: weight 0
+    {
+        const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
+        const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
+        for (int k = 0; k < g.NS; ++k) {
+            TZ* zs = reinterpret_cast<TZ*>(dsm + (size_t)k * stage);
+            for (int t = lenc + tid; t < kSW * g.Lw + kZPer; t += kSThreads) zs[t] = neg_inf<TZ>();
         }
     }
-    const int rows_g = grp < P.rows ? (P.rows - grp + g.G - 1) / g.G : 0;
-    const float inv_n = 1.f / (float)P.N;
-    constexpr int kZPer = 16 / (int)sizeof(TZ);          // logits per 16 bytes
 
-    // ---- this warp's segment, its kept tokens, its share of shared memory -------------------------
-    const int cw = warp < kSW ? warp : 0;                // the exchange warp owns no segment
-    const int seg = crank * kSW + cw;
-    const long long j0l = (long long)seg * g.Lw;
-    const int j0 = (int)(j0l < P.N ? j0l : P.N);
-    const int len = max(0, min(P.N - j0, g.Lw));
-    const int len_v = len & ~(kZPer - 1);
-    const uint32_t zbytes = (uint32_t)len_v * (uint32_t)sizeof(TZ);
-    const int r_lo = rank_at(P, j0, n_valid), r_hi = rank_at(P, j0 + len, n_valid);
-    const int kc = r_hi - r_lo;
-    const int dummy = r_lo & 1;            // slot 0 of the warp's pair grid belongs to the previous segment
-    const int r0 = r_lo - dummy;           // drafter index of slot 0
-    const int kcp = kc + dummy;            // slots in use
-    const int kcs = min(kcp, g.ycap);      // ... of which staged and cached
-    const int nsteps = (kcs + 63) >> 6;    // steps of 32 lanes x 2 slots
-
-    const size_t off_y = (size_t)kSW * g.NS * g.zstage;
-    const size_t off_cache = off_y + (size_t)kSW * g.NS * g.ystage;
-    const size_t off_goff = off_cache + (size_t)kSW * 2 * g.ycap * 8;
-    const size_t off_bar = off_goff + (size_t)kSW * g.ycap * 2;
-    const uint32_t dsm_a = smem_u32(dsm);
-    const uint32_t zst_a = dsm_a + (uint32_t)(cw * g.NS * g.zstage);
-    const uint32_t yst_a = dsm_a + (uint32_t)(off_y + (size_t)cw * g.NS * g.ystage);
-    const uint32_t cache_a = dsm_a + (uint32_t)(off_cache + (size_t)cw * 2 * g.ycap * 8);
-    const uint32_t goff_a = dsm_a + (uint32_t)(off_goff + (size_t)cw * g.ycap * 2);
-    const uint32_t bar_a = dsm_a + (uint32_t)(off_bar + (size_t)cw * g.NS * 8);
-    unsigned char* zst_p = dsm + (size_t)cw * g.NS * g.zstage;
-    unsigned char* yst_p = dsm + off_y + (size_t)cw * g.NS * g.ystage;
-
+    // streaming warp w: its own segment; exchange and load warp: lane w looks after warp w's segment
+    const int seg = crank * kSW + (warp < kSW ? warp : (lane & (kSW - 1)));
+    const SegInfo si = seg_info(P, g, seg, n_valid);
     if (warp < kSW) {
-        if (lane == 0)
-            for (int s = 0; s < g.NS; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a + 8u * s));
-        // beyond the segment (and the 16 spare bytes of every stage): weight 0
-        for (int s = 0; s < g.NS; ++s) {
-            TZ* zs = reinterpret_cast<TZ*>(zst_p + (size_t)s * g.zstage);
-            for (int t = len + lane; t < g.ST + kZPer; t += 32) zs[t] = neg_inf<TZ>();
-        }
-        // shared byte offset (within a stage, 16 bits) of the target logit of every cached slot; unused
-        // slots point at the spare -inf
-        uint32_t* goff_p = reinterpret_cast<uint32_t*>(dsm + off_goff + (size_t)cw * g.ycap * 2);
-        const uint32_t spare = (uint32_t)g.ST * (uint32_t)sizeof(TZ);
-        for (int q = lane; q < nsteps * 32; q += 32) {
-            uint32_t o[2];
+        // ================================ streaming warps ============================================
+        const int r0 = si.r0, kcs = si.kcs, j0 = si.j0;
+        const int nsteps = (kcs + 63) >> 6;                 // steps of 32 lanes x 2 slots
+        const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);   // the warp's segment within the slice
+        // shared byte offset (from the start of the slice, 16 bits) of the target logit of every cached
+        // slot; slots that hold no kept token of this segment point at the spare -inf
+        {
+            uint32_t* goff_p = reinterpret_cast<uint32_t*>(dsm + off_goff + (size_t)warp * g.ycap * 2);
+            for (int q = lane; q < nsteps * 32; q += 32) {
+                uint32_t o[2];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int il = 2 * q + h;
-                o[h] = spare;
-                if (il < kcs && !(dummy && il == 0)) o[h] = (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ);
+                for (int h = 0; h < 2; ++h) {
+                    const int il = 2 * q + h;
+                    o[h] = zslice;
+                    if (il < kcs && !(si.dummy && il == 0))
+                        o[h] = zw_off + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ);
+                }
+                goff_p[q] = o[0] | (o[1] << 16);
             }
-            goff_p[q] = o[0] | (o[1] << 16);
         }
     }
-    if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
-    if (warp == kSW) {
-        // ---- exchange warp: per row, fold the CTA's 16 warp records into one, publish it, collect the
-        // ---- C records of the row and leave the row scalars in shared memory, ahead of the second visits
+    if (warp < kSW) {
+        const int r0 = si.r0, kcp = si.kcp, kcs = si.kcs, j0 = si.j0;
+        const int nsteps = (kcs + 63) >> 6;
+        const bool ovf = kcp > kcs;
+        const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
+        const uint32_t yw_off = zslice + 16u + (uint32_t)warp * (uint32_t)g.ystage;
+        const uint32_t csz = (uint32_t)g.ycap * 8u;
+        const uint32_t cb0 = dsm_a + off_cache + (uint32_t)warp * 2u * csz + (uint32_t)lane * 16u;
+        const uint32_t gl = dsm_a + off_goff + (uint32_t)warp * (uint32_t)g.ycap * 2u + (uint32_t)lane * 4u;
+        // this lane's slots of the pair grid that hold no kept token of the segment (slot 0 when it belongs
+        // to the previous segment, and the tail of the last step), as element indices, -1 = none
+        const int pad_a = (si.dummy && lane == 0 && kcs > 0) ? 0 : -1;
+        const int pad_b = kcs + lane < nsteps * 64 ? kcs + lane : -1;
+        const int pad_c = kcs + lane + 32 < nsteps * 64 ? kcs + lane + 32 : -1;
+        const long long ystep = (long long)g.G * P.drafter_stride;
+        const float2 l2e = splat(kLog2e);
+
+        // ---- second visit of local row `itb`: sum of min(p, q~) over the cached kept tokens -----------
+        auto second_visit = [&](int itb) {
+            const int par = itb & 1;
+            mbar_wait(smem_u32(&rbar[par]), (uint32_t)((itb >> 1) & 1), &fail);
+            const float theta = scal[par][4];
+            const float2 f = fzy[par][warp];                  // p = f.x e_z,  q' = f.y e_y
+            // q~ = q' + x (theta - q'),  x = p / N
+            const float2 fz2 = splat(f.x), fy2 = splat(f.y), xs2 = splat(f.x * inv_n), th2 = splat(theta), neg1 = splat(-1.f);
+            float2 ak2 = splat(0.f);
+            const uint32_t cb = cb0 + (uint32_t)par * csz;
+#pragma unroll 2
+            for (int st = 0; st < nsteps; ++st) {
+                const uint4 c4 = lds128(cb + (uint32_t)st * 512u);
+                const float2 ez = make_float2(__uint_as_float(c4.x), __uint_as_float(c4.y));
+                const float2 ey = make_float2(__uint_as_float(c4.z), __uint_as_float(c4.w));
+                const float2 p = fmul2(ez, fz2), qp = fmul2(ey, fy2), x = fmul2(ez, xs2);
+                const float2 w = ffma2(x, ffma2(qp, neg1, th2), qp);
+                ak2 = fadd2(ak2, make_float2(fminf(p.x, w.x), fminf(p.y, w.y)));
+            }
+            float ak = ak2.x + ak2.y;
+            if (ovf) {   // kept tokens beyond the cache: from global memory again
+                const long long row = grp + (long long)itb * g.G;
+                const TZ* zrow = static_cast<const TZ*>(P.target) + row * P.target_stride;
+                const TY* yrow = static_cast<const TY*>(P.drafter) + row * P.drafter_stride;
+                const float m_w = wrec[par][warp][4], my_w = wrec[par][warp][5];
+                const float zoff = m_w > -INFINITY ? -m_w * kLog2e : 0.f, yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
+                for (int il = kcs + lane; il < kcp; il += 32) {
+                    const float ez = ex2(fmaf(to_float<TZ>(zrow[__ldg(P.ids + r0 + il)]), kLog2e, zoff));
+                    const float y = to_float<TY>(yrow[r0 + il]);
+                    const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
+                    const float p = ez * f.x, qp = ey * f.y;
+                    ak += fminf(p, fmaf(p * inv_n, theta - qp, qp));
+                }
+            }
+            ak = warp_sum(ak);
+            if (lane == 0) {
+                akv[par][warp] = ak;
+                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bbar[par])) : "memory");
+            }
+        };
+
+        // ---- main loop: first visit of row it, second visit of row it - 1 -------------------------------
+        const TY* cy = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + r0;   // slot 0 of the current row
+        int s = 0;
+        uint32_t sph = 0, st_a = dsm_a, fb = full_a, eb = empty_a;
+        unsigned char* st_p = dsm;
+        for (int it = 0; it < rows_g; ++it) {
+            const int par = it & 1;
+            const uint32_t zs_a = st_a + zw_off;
+            const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(cy) & 15u);      // slot 0 sits this many bytes into the warp's region
+            const uint32_t ys_a = st_a + yw_off + shb + (uint32_t)lane * 2u * (uint32_t)sizeof(TY);   // this lane's pair of step 0
+            mbar_wait(fb, sph, &fail);
+
+            // slots that hold no kept token of this segment read as weight 0
+            {
+                TY* yp = reinterpret_cast<TY*>(st_p + yw_off + shb);
+                const TY fill = KIND == RDK_LOGITS ? neg_inf<TY>() : zero_of<TY>();
+                if (pad_a >= 0) yp[pad_a] = fill;
+                if (pad_b >= 0) yp[pad_b] = fill;
+                if (pad_c >= 0) yp[pad_c] = fill;
+                __syncwarp();
+            }
+
+            // maxima of the segment and of its kept drafter values
+            uint4 zv[NIT > 0 ? NIT : 1];
+            MaxAcc<TZ> mz;
+            if (NIT > 0) {
+#pragma unroll
+                for (int k = 0; k < NIT; ++k) zv[k] = lds128(zs_a + (uint32_t)(k * 32 + lane) * 16u);
+#pragma unroll
+                for (int k = 0; k < NIT; ++k) mz.push(zv[k]);
+            } else {
+#pragma unroll 4
+                for (int t = lane * kZPer; t < g.Lw; t += 32 * kZPer) mz.push(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)));
+            }
+            float my_w = KIND == RDK_LOGITS ? -INFINITY : 0.f;
+            if (KIND == RDK_LOGITS) {
+#pragma unroll 2
+                for (int st = 0; st < nsteps; ++st) {
+                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)st * 64u * (uint32_t)sizeof(TY));
+                    my_w = fmaxf(my_w, fmaxf(y.x, y.y));
+                }
+                if (ovf)
+                    for (int il = kcs + lane; il < kcp; il += 32) my_w = fmaxf(my_w, to_float<TY>(cy[il]));
+                my_w = warp_max_redux(my_w);
+            }
+            const float m_w = warp_max_redux(mz.result());
+            const float zoff = m_w > -INFINITY ? -m_w * kLog2e : 0.f;
+            const float yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
+
+            // soft-max sweep: sum of e over the segment
+            float2 Ea = splat(0.f), Eb = splat(0.f);
+            {
+                const float2 of = splat(zoff);
+                if (NIT > 0) {
+#pragma unroll
+                    for (int k = 0; k < NIT; ++k) exp_sum_vec<TZ>(zv[k], l2e, of, Ea, Eb);
+                } else {
+#pragma unroll 4
+                    for (int t = lane * kZPer; t < g.Lw; t += 32 * kZPer)
+                        exp_sum_vec<TZ>(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)), l2e, of, Ea, Eb);
+                }
+            }
+            // kept tokens: e_z, e_y, their sums; the pairs go to the cache
+            float2 K1 = splat(0.f), Zq = splat(0.f), th = splat(0.f);
+            {
+                const float2 zof = splat(zoff), yof = splat(yoff);
+                const uint32_t cb = cb0 + (uint32_t)par * csz;
+#pragma unroll 2
+                for (int st = 0; st < nsteps; ++st) {
+                    const uint32_t go = lds32(gl + (uint32_t)st * 128u);
+                    const float2 z = make_float2(lds_z<TZ>(st_a + (go & 0xffffu)), lds_z<TZ>(st_a + (go >> 16)));
+                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)st * 64u * (uint32_t)sizeof(TY));
+                    const float2 ez = ex2_2(ffma2(z, l2e, zof));
+                    const float2 ey = KIND == RDK_LOGITS ? ex2_2(ffma2(y, l2e, yof)) : y;
+                    K1 = fadd2(K1, ez); Zq = fadd2(Zq, ey); th = ffma2(ez, ey, th);
+                    sts128(cb + (uint32_t)st * 512u, ez.x, ez.y, ey.x, ey.y);
+                }
+            }
+            float E1s = (Ea.x + Ea.y) + (Eb.x + Eb.y), K1s = K1.x + K1.y, Zqs = Zq.x + Zq.y, ths = th.x + th.y;
+            if (ovf) {
+                for (int il = kcs + lane; il < kcp; il += 32) {               // kept tokens beyond the cache
+                    const float ez = ex2(fmaf(lds_z<TZ>(zs_a + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ)), kLog2e, zoff));
+                    const float y = to_float<TY>(cy[il]);
+                    const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
+                    K1s += ez; Zqs += ey; ths = fmaf(ez, ey, ths);
+                }
+            }
+            const float tot = warp_sum4(E1s, K1s, Zqs, ths, lane);      // lanes 0, 8, 16, 24 hold the four totals
+            // the warp's record goes to the exchange warp, the stage back to the load warp
+            if ((lane & 7) == 0) wrec[par][warp][lane >> 3] = tot;
+            if (lane == 0) *reinterpret_cast<float2*>(&wrec[par][warp][4]) = make_float2(m_w, my_w);
+            __syncwarp();
+            if (lane == 0) {
+                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&abar[par])) : "memory");
+                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(eb) : "memory");
+            }
+
+            if (it > 0) second_visit(it - 1);
+            cy += ystep;
+            st_a += stage; st_p += stage; fb += 8u; eb += 8u;
+            if (++s == g.NS) { s = 0; sph ^= 1u; st_a = dsm_a; st_p = dsm; fb = full_a; eb = empty_a; }
+        }
+        if (rows_g > 0) second_visit(rows_g - 1);
+    } else if (warp == kSW) {
+        // ================================ exchange warp =================================================
+        // per row: fold the CTA's 16 warp records into one and publish it; collect the C records of the
+        // row; leave the row scalars and every warp's factors in shared memory for the second visits;
+        // and turn the previous row's second-visit sums into the per-segment sums the draw kernel reads
+        // lane w < 16 keeps warp w's sums and factors of the row whose second visit is pending in
+        // registers (the shared copies are overwritten two rows on, possibly before that visit ends)
+        float4 w0 = make_float4(0.f, 0.f, 0.f, 0.f);
+        float2 f = make_float2(0.f, 0.f);
+        float theta = 0.f;
+        auto finish_row = [&](int itf) {       // lane w < 16: segment sums of warp w
+            const int pf = itf & 1;
+            const long long row = grp + (long long)itf * g.G;
+            mbar_wait(smem_u32(&bbar[pf]), (uint32_t)((itf >> 1) & 1), &fail);
+            if (lane < kSW) {
+                const float ak = akv[pf][lane];
+                // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
+                const float segP = w0.x * f.x;
+                const float xs = f.x * inv_n;
+                const float oov = theta * xs * fmaxf(0.f, w0.x - w0.y);
+                const float Kw = f.y * w0.z - f.y * xs * w0.w + theta * xs * w0.y;
+                const float a_s = oov + ak;
+                reinterpret_cast<float4*>(P.rec + row * kRecFloats + 16)[seg] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP - a_s), segP);
+            }
+        };
         for (int it = 0; it < rows_g; ++it) {
             const int par = it & 1;
             const uint32_t ph = (uint32_t)((it >> 1) & 1);
             const long long row = grp + (long long)it * g.G;
             mbar_wait(smem_u32(&abar[par]), ph, &fail);
-            float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY;
+            float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY, K1 = 0.f;
             if (lane < kSW) {
                 const volatile float* wr = &wrec[par][lane][0];
-                E1 = wr[0]; Zq = wr[2]; th = wr[3]; m = wr[4]; my = wr[5];
+                E1 = wr[0]; K1 = wr[1]; Zq = wr[2]; th = wr[3]; m = wr[4]; my = wr[5];
             }
-            combine_records(E1, Zq, th, m, my);
+            const float4 w_now = make_float4(E1, K1, Zq, th);
+            const float m_w = m, my_w = my;
+            combine_records(E1, Zq, th, m, my, lane);
             if (lane == 0) {
                 unsigned char* xr = P.xrec + ((size_t)row * g.C + crank) * kXrecBytes;
                 st_tagged(xr, E1, g.tag); st_tagged(xr + 8, Zq, g.tag); st_tagged(xr + 16, th, g.tag);
                 st_tagged(xr + 24, m, g.tag); st_tagged(xr + 32, my, g.tag);
             }
+            if (it > 0) finish_row(it - 1);
             E1 = 0.f; Zq = 0.f; th = 0.f; m = -INFINITY; my = -INFINITY;
             if (lane < g.C) {
                 const unsigned char* xr = P.xrec + ((size_t)row * g.C + lane) * kXrecBytes;
@@ -384,222 +593,80 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 E1 = __uint_as_float((uint32_t)w[0]); Zq = __uint_as_float((uint32_t)w[1]); th = __uint_as_float((uint32_t)w[2]);
                 m = __uint_as_float((uint32_t)w[3]); my = __uint_as_float((uint32_t)w[4]);
             }
-            combine_records(E1, Zq, th, m, my);
+            combine_records(E1, Zq, th, m, my, lane);
             const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
-            const float theta = th * inv_zp * inv_zq;
+            theta = th * inv_zp * inv_zq;
+            w0 = w_now;
+            f.x = (m_w > -INFINITY ? ex2((m_w - m) * kLog2e) : 0.f) * inv_zp;
+            f.y = (KIND == RDK_LOGITS ? (my_w > -INFINITY ? ex2((my_w - my) * kLog2e) : 0.f) : 1.f) * inv_zq;
+            if (lane < kSW) fzy[par][lane] = f;
             if (lane == 0) {
                 float* sc = scal[par];
-                sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq;
-                sc[4] = theta; sc[5] = m; sc[6] = my;
+                sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq; sc[4] = theta;
                 if (crank == 0) {
                     float* rec = P.rec + row * kRecFloats;
                     rec[kRecOffg] = sc[0]; rec[kRecInvZp] = inv_zp; rec[kRecYoffg] = sc[2]; rec[kRecInvZq] = inv_zq;
                     rec[kRecTheta] = theta; rec[kRecInvN] = inv_n; rec[kRecInvS] = 1.f; rec[kRecS] = 1.f;
                 }
-                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[par])) : "memory");
             }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[par])) : "memory");
             if (crank == 0 && P.counters && row % P.positions == 0)
                 for (int t = lane; t < P.trials; t += 32) P.counters[(row / P.positions) * P.trials + t] = 0;
         }
+        if (rows_g > 0) finish_row(rows_g - 1);
     } else {
-        // ---- streaming warps ---------------------------------------------------------------------------
-        const long long zstep = (long long)g.G * P.target_stride, ystep = (long long)g.G * P.drafter_stride;
+        // ================================ load warp =====================================================
+        // per row: one bulk copy of the CTA's slice of the target row and one per warp of the matching
+        // drafter values, into the stage the streaming warps have released
+        const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
+        const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
+        const int lenc_v = lenc & ~(kZPer - 1);
+        const uint32_t zbytes = (uint32_t)lenc_v * (uint32_t)sizeof(TZ);
+        const uint32_t kbytes = lane < kSW ? (uint32_t)si.kcs * (uint32_t)sizeof(TY) : 0u;
         const uintptr_t y_end16 = reinterpret_cast<uintptr_t>(static_cast<const TY*>(P.drafter) +
                                                               (long long)(P.rows - 1) * P.drafter_stride + P.n) & ~uintptr_t(15);
-        // next row to load, and the stage it goes to
-        const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0;
-        const TY* ny = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + r0;
-        int is = 0;
-        // Loads of one row into stage `is`.  Lanes stage the few elements a 16-byte bulk copy cannot
-        // cover with plain stores, then lane 0 arms the barrier and starts the copies.
-        auto issue_next = [&]() {
-            TZ* zs = reinterpret_cast<TZ*>(zst_p + (size_t)is * g.zstage);
-            unsigned char* ys = yst_p + (size_t)is * g.ystage;
-            const uintptr_t b0 = reinterpret_cast<uintptr_t>(ny), b1 = b0 + (uintptr_t)kcs * sizeof(TY);
+        const long long zstep = (long long)g.G * P.target_stride, ystep = (long long)g.G * P.drafter_stride;
+        const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0c;
+        const TY* ny = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + si.r0;
+        const uint32_t yw_off = zslice + 16u + (uint32_t)(lane & (kSW - 1)) * (uint32_t)g.ystage;
+        int s = 0;
+        uint32_t eph = 1, st_a = dsm_a, fb = full_a, eb = empty_a;    // a fresh stage counts as released
+        unsigned char* st_p = dsm;
+        for (int it = 0; it < rows_g; ++it) {
+            mbar_wait(eb, eph, &fail);
+            // the few elements a 16-byte copy cannot cover go by plain stores: a slice that ends inside a
+            // vector, and the very end of the drafter buffer
+            const uintptr_t b0 = reinterpret_cast<uintptr_t>(ny), b1 = b0 + kbytes;
             const uintptr_t a0 = b0 & ~uintptr_t(15);
             uintptr_t a1 = (b1 + 15) & ~uintptr_t(15);
             if (a1 > y_end16) a1 = y_end16 > a0 ? y_end16 : a0;     // never read past the drafter buffer
-            const uint32_t ybytes = kcs ? (uint32_t)(a1 - a0) : 0u;
-            if (len > len_v) {
-                if (lane < len - len_v) zs[len_v + lane] = nz[len_v + lane];
-            }
-            if (kcs && a1 < b1) {
+            const uint32_t ybytes = kbytes ? (uint32_t)(a1 - a0) : 0u;
+            if (lane < lenc - lenc_v) reinterpret_cast<TZ*>(st_p)[lenc_v + lane] = nz[lenc_v + lane];
+            if (kbytes && a1 < b1) {
                 const uintptr_t t0 = a1 > b0 ? a1 : b0;
                 const int nt = (int)((b1 - t0) / sizeof(TY));
-                if (lane < nt) reinterpret_cast<TY*>(ys + (t0 - a0))[lane] = reinterpret_cast<const TY*>(t0)[lane];
+                for (int k = 0; k < nt; ++k) reinterpret_cast<TY*>(st_p + yw_off + (t0 - a0))[k] = reinterpret_cast<const TY*>(t0)[k];
             }
-            __syncwarp();
+            const uint32_t total = zbytes + __reduce_add_sync(0xffffffffu, ybytes);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage was last touched by plain loads and stores
             if (lane == 0) {
-                const uint32_t bar = bar_a + 8u * is;
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                if (zbytes + ybytes == 0) {
-                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-                } else {
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(zbytes + ybytes) : "memory");
-                    if (zbytes)
-                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                     ::"r"(zst_a + (uint32_t)(is * g.zstage)), "l"(nz), "r"(zbytes), "r"(bar) : "memory");
-                    if (ybytes)
-                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                     ::"r"(yst_a + (uint32_t)(is * g.ystage)), "l"(a0), "r"(ybytes), "r"(bar) : "memory");
+                if (total == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(fb) : "memory");
+                else asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(total) : "memory");
+                for (uint32_t off = 0; off < zbytes; off += 32768u) {
+                    const uint32_t sz = min(32768u, zbytes - off);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(st_a + off), "l"(reinterpret_cast<const char*>(nz) + off), "r"(sz), "r"(fb) : "memory");
                 }
             }
+            __syncwarp();
+            if (ybytes)
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(st_a + yw_off), "l"(a0), "r"(ybytes), "r"(fb) : "memory");
             nz += zstep; ny += ystep;
-            is = is + 1 == g.NS ? 0 : is + 1;
-        };
-        for (int itx = 0; itx < g.NS && itx < rows_g; ++itx) issue_next();
-
-        const float2 l2e = splat(kLog2e);
-
-        // ---- second visit of local row `itb` -----------------------------------------------------
-        auto second_visit = [&](int itb) {
-            const int par = itb & 1;
-            const long long row = grp + (long long)itb * g.G;
-            mbar_wait(smem_u32(&rbar[par]), (uint32_t)((itb >> 1) & 1), &fail);
-            const float4 s0 = *reinterpret_cast<const float4*>(&scal[par][0]);   // -m log2e, 1/Zp, -my log2e, 1/Zq
-            const float4 s1 = *reinterpret_cast<const float4*>(&scal[par][4]);   // theta, m, my
-            const float4 w0 = *reinterpret_cast<const float4*>(&wrec[par][warp][0]);   // this warp's sums of the row
-            const float2 w1 = *reinterpret_cast<const float2*>(&wrec[par][warp][4]);   // ... and maxima
-            const float theta = s1.x;
-            const float fz = (w1.x > -INFINITY ? ex2((w1.x - s1.y) * kLog2e) : 0.f) * s0.y;
-            const float fy = (KIND == RDK_LOGITS ? (w1.y > -INFINITY ? ex2((w1.y - s1.z) * kLog2e) : 0.f) : 1.f) * s0.w;
-            // kept tokens: sum of min(p, q~), q~ = q' + x (theta - q'), from the cached (e_z, e_y)
-            const float2 fz2 = splat(fz), fy2 = splat(fy), xs2 = splat(fz * inv_n), th2 = splat(theta), neg1 = splat(-1.f);
-            float2 ak2 = splat(0.f);
-            const uint32_t cb = cache_a + (uint32_t)(par * g.ycap * 8) + (uint32_t)lane * 16u;
-#pragma unroll 4
-            for (int st = 0; st < nsteps; ++st) {
-                const uint4 c4 = lds128(cb + (uint32_t)st * 512u);
-                const float2 ez = make_float2(__uint_as_float(c4.x), __uint_as_float(c4.y));
-                const float2 ey = make_float2(__uint_as_float(c4.z), __uint_as_float(c4.w));
-                const float2 p = fmul2(ez, fz2), qp = fmul2(ey, fy2), x = fmul2(ez, xs2);
-                const float2 w = ffma2(x, ffma2(qp, neg1, th2), qp);
-                ak2 = fadd2(ak2, make_float2(fminf(p.x, w.x), fminf(p.y, w.y)));
-            }
-            float ak = ak2.x + ak2.y;
-            if (kcp > kcs) {   // kept tokens beyond the cache: from global memory again
-                const TZ* zrow = static_cast<const TZ*>(P.target) + row * P.target_stride;
-                const TY* yrow = static_cast<const TY*>(P.drafter) + row * P.drafter_stride;
-                const float zoff = w1.x > -INFINITY ? -w1.x * kLog2e : 0.f, yoff = w1.y > -INFINITY ? -w1.y * kLog2e : 0.f;
-                for (int il = kcs + lane; il < kcp; il += 32) {
-                    const float ez = ex2(fmaf(to_float<TZ>(zrow[__ldg(P.ids + r0 + il)]), kLog2e, zoff));
-                    const float y = to_float<TY>(yrow[r0 + il]);
-                    const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
-                    const float p = ez * fz, qp = ey * fy;
-                    ak += fminf(p, fmaf(p * inv_n, theta - qp, qp));
-                }
-            }
-            ak = warp_sum(ak);
-            if (lane == 0) {
-                // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
-                const float segP = w0.x * fz;
-                const float oov = theta * inv_n * fmaxf(0.f, w0.x - w0.y) * fz;
-                const float xs = fz * inv_n;
-                const float Kw = fy * w0.z - fy * xs * w0.w + theta * xs * w0.y;
-                const float a_s = oov + ak;
-                reinterpret_cast<float4*>(P.rec + row * kRecFloats + 16)[seg] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP - a_s), segP);
-            }
-        };
-
-        // ---- main loop: first visit of row it, reload of its stage, second visit of row it - 1 ----
-        const TY* cy = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + r0;   // slot 0 of the current row
-        int s = 0;
-        uint32_t sph = 0;
-        for (int it = 0; it < rows_g; ++it) {
-            const int par = it & 1;
-            const uint32_t zs_a = zst_a + (uint32_t)(s * g.zstage);
-            const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(cy) & 15u);      // slot 0 sits this many bytes into the stage
-            const uint32_t ys_a = yst_a + (uint32_t)(s * g.ystage) + shb;
-            mbar_wait(bar_a + 8u * s, sph, &fail);
-
-            // slots of the pair grid that hold no kept token of this segment read as weight 0
-            {
-                TY* yp = reinterpret_cast<TY*>(yst_p + (size_t)s * g.ystage + shb);
-                const TY fill = KIND == RDK_LOGITS ? neg_inf<TY>() : zero_of<TY>();
-                if (dummy && lane == 0 && kcs > 0) yp[0] = fill;
-                for (int il = kcs + lane; il < nsteps * 64; il += 32) yp[il] = fill;
-                __syncwarp();
-            }
-
-            // maxima of the segment and of its kept drafter values
-            uint4 zv[NIT > 0 ? NIT : 1];
-            MaxAcc<TZ> mz;
-            if (NIT > 0) {
-#pragma unroll
-                for (int k = 0; k < NIT; ++k) zv[k] = lds128(zs_a + (uint32_t)(k * 32 + lane) * 16u);
-#pragma unroll
-                for (int k = 0; k < NIT; ++k) mz.push(zv[k]);
-            } else {
-#pragma unroll 4
-                for (int t = lane * kZPer; t < g.ST; t += 32 * kZPer) mz.push(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)));
-            }
-            float my_w = KIND == RDK_LOGITS ? -INFINITY : 0.f;
-            if (KIND == RDK_LOGITS) {
-#pragma unroll 4
-                for (int st = 0; st < nsteps; ++st) {
-                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)(st * 64 + lane * 2) * (uint32_t)sizeof(TY));
-                    my_w = fmaxf(my_w, fmaxf(y.x, y.y));
-                }
-                for (int il = kcs + lane; il < kcp; il += 32) my_w = fmaxf(my_w, to_float<TY>(cy[il]));
-                my_w = warp_max_redux(my_w);
-            }
-            const float m_w = warp_max_redux(mz.result());
-            const float zoff = m_w > -INFINITY ? -m_w * kLog2e : 0.f;
-            const float yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
-
-            // soft-max sweep: sum of e over the segment
-            float2 Ea = splat(0.f), Eb = splat(0.f);
-            {
-                const float2 of = splat(zoff);
-                if (NIT > 0) {
-#pragma unroll
-                    for (int k = 0; k < NIT; ++k) exp_sum_vec<TZ>(zv[k], l2e, of, Ea, Eb);
-                } else {
-#pragma unroll 4
-                    for (int t = lane * kZPer; t < g.ST; t += 32 * kZPer)
-                        exp_sum_vec<TZ>(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)), l2e, of, Ea, Eb);
-                }
-            }
-            // kept tokens: e_z, e_y, their sums; the pairs go to the cache
-            float2 K1 = splat(0.f), Zq = splat(0.f), th = splat(0.f);
-            {
-                const float2 zof = splat(zoff), yof = splat(yoff);
-                const uint32_t cb = cache_a + (uint32_t)(par * g.ycap * 8) + (uint32_t)lane * 16u;
-#pragma unroll 2
-                for (int st = 0; st < nsteps; ++st) {
-                    const uint32_t go = lds32(goff_a + (uint32_t)(st * 32 + lane) * 4u);
-                    const float2 z = make_float2(lds_z<TZ>(zs_a + (go & 0xffffu)), lds_z<TZ>(zs_a + (go >> 16)));
-                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)(st * 64 + lane * 2) * (uint32_t)sizeof(TY));
-                    const float2 ez = ex2_2(ffma2(z, l2e, zof));
-                    const float2 ey = KIND == RDK_LOGITS ? ex2_2(ffma2(y, l2e, yof)) : y;
-                    K1 = fadd2(K1, ez); Zq = fadd2(Zq, ey); th = ffma2(ez, ey, th);
-                    sts128(cb + (uint32_t)st * 512u, ez.x, ez.y, ey.x, ey.y);
-                }
-            }
-            float E1s = (Ea.x + Ea.y) + (Eb.x + Eb.y), K1s = K1.x + K1.y, Zqs = Zq.x + Zq.y, ths = th.x + th.y;
-            for (int il = kcs + lane; il < kcp; il += 32) {               // kept tokens beyond the cache
-                const float ez = ex2(fmaf(lds_z<TZ>(zs_a + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ)), kLog2e, zoff));
-                const float y = to_float<TY>(cy[il]);
-                const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
-                K1s += ez; Zqs += ey; ths = fmaf(ez, ey, ths);
-            }
-            const float tot = warp_sum4(E1s, K1s, Zqs, ths, lane);      // lanes 0, 8, 16, 24 hold the four totals
-
-            // the stage is free: bring in the row NS ahead
-            __syncwarp();
-            if (it + g.NS < rows_g) issue_next();
-
-            // hand the warp's record to the exchange warp
-            if ((lane & 7) == 0) wrec[par][warp][lane >> 3] = tot;
-            if (lane == 0) { wrec[par][warp][4] = m_w; wrec[par][warp][5] = my_w; }
-            __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&abar[par])) : "memory");
-
-            if (it > 0) second_visit(it - 1);
-            cy += ystep;
-            if (++s == g.NS) { s = 0; sph ^= 1u; }
+            st_a += stage; st_p += stage; fb += 8u; eb += 8u;
+            if (++s == g.NS) { s = 0; eph ^= 1u; st_a = dsm_a; st_p = dsm; fb = full_a; eb = empty_a; }
         }
-        if (rows_g > 0) second_visit(rows_g - 1);
     }
     __syncthreads();
     if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
@@ -795,22 +862,22 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-static size_t stream_smem(const StreamGeo& g) {
-    return (size_t)kSW * ((size_t)g.NS * (g.zstage + g.ystage + 8) + (size_t)g.ycap * 18);   // + cache (2 x 8 bytes) and offsets (2 bytes) per slot
+static size_t stream_smem(const StreamGeo& g, size_t es) {
+    const size_t stage = (size_t)kSW * g.Lw * es + 16 + (size_t)kSW * g.ystage;
+    return (size_t)g.NS * stage + (size_t)kSW * g.ycap * 18 + (size_t)g.NS * 16;   // + cache (2 x 8 bytes) and offsets (2 bytes) per slot, barriers
 }
 
 // Group size, segment length, stage count and cache capacity for a vocabulary of N tokens with n
 // kept ids; false when the shapes do not fit shared memory.
 static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
     const size_t budget = 225 * 1024;      // dynamic shared memory a CTA may ask for, less the static part
-    int C = (N + kSW * 1024 - 1) / (kSW * 1024);
+    const int vt = 32 * (int)(16 / es);    // tokens one warp covers with one 16-byte vector per lane
+    int C = (N + kSW * 4 * vt - 1) / (kSW * 4 * vt);
     if (C > kMaxGroup) C = kMaxGroup;
-    const int per = (N + C * kSW - 1) / (C * kSW);
     g.C = C;
-    g.Lw = (per + 7) & ~7;
-    g.ST = (g.Lw + 255) & ~255;
-    g.zstage = g.ST * (int)es + 16;
-    if ((g.Lw + kSeg - 1) / kSeg > kMaxChunks || g.zstage > 65535) return false;   // stage offsets are 16-bit
+    g.nv = (N + C * kSW * vt - 1) / (C * kSW * vt);
+    g.Lw = g.nv * vt;
+    if ((g.Lw + kSeg - 1) / kSeg > kMaxChunks || (size_t)kSW * g.Lw * es + 16 > 65535) return false;   // slice offsets are 16-bit
     const long long expect = ((long long)n * g.Lw + N - 1) / N;
     long long cap = expect + expect / 8 + 32;
     const long long most = (long long)(n < g.Lw ? n : g.Lw) + 1;
@@ -821,7 +888,7 @@ static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
         while (c >= 64) {
             g.ycap = (int)c;
             g.ystage = (int)((((size_t)c + 16) * ys + 15) & ~size_t(15));
-            if (stream_smem(g) <= budget) return true;
+            if (stream_smem(g, es) <= budget) return true;
             if (g.NS > 2) break;          // first give up a stage, then cache capacity
             c -= 64;
         }
@@ -832,7 +899,7 @@ static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
 template <typename TZ, typename TY, int KIND, int NIT>
 static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s) {
     auto kern = rdk_stream_kernel<TZ, TY, KIND, NIT>;
-    const size_t smem = stream_smem(g);
+    const size_t smem = stream_smem(g, sizeof(TZ));
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // how many CTAs are resident at once (cached per kernel instance, shared-memory size and device)
@@ -880,8 +947,8 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
 
 template <typename TZ, typename TY, int KIND>
 static cudaError_t launch_nit(const RowParams& P, const StreamGeo& g, cudaStream_t s) {
-    // the common stage length (four 16-byte vectors per lane) gets the register-resident sweep
-    if (g.ST == 4 * 32 * (16 / (int)sizeof(TZ))) return launch_stream<TZ, TY, KIND, 4>(P, g, s);
+    // the common segment length (four 16-byte vectors per lane) gets the register-resident sweep
+    if (g.nv == 4) return launch_stream<TZ, TY, KIND, 4>(P, g, s);
     return launch_stream<TZ, TY, KIND, 0>(P, g, s);
 }
 
