@@ -292,7 +292,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     __shared__ __align__(8) unsigned long long bbar[2];   // [row parity]: akv[] of the row is set
     __shared__ int fail;
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);     // the same in every lane, and the compiler knows it
     const int grp = blockIdx.x / g.C, crank = blockIdx.x % g.C;
 
     if (!index_matches(P)) {   // same decision in every CTA of the grid; nothing is in flight yet
@@ -372,7 +373,9 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     __syncthreads();
 
     if (warp < kSW) {
-        const int r0 = si.r0, kcp = si.kcp, kcs = si.kcs, j0 = si.j0;
+        // per-warp quantities, taken from lane 0 so that loops over them are not treated as divergent
+        const int r0 = __shfl_sync(0xffffffffu, si.r0, 0), kcp = __shfl_sync(0xffffffffu, si.kcp, 0);
+        const int kcs = __shfl_sync(0xffffffffu, si.kcs, 0), j0 = __shfl_sync(0xffffffffu, si.j0, 0);
         const int nsteps = (kcs + 63) >> 6;
         const bool ovf = kcp > kcs;
         const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
