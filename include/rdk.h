@@ -206,10 +206,14 @@ int rdk_redistribute_linear(const rdk_problem* problem, const void* target, cons
  *   out        see rdk_outputs
  *   ws         device workspace of rdk_sample_workspace_bytes(problem, mode, trials) bytes, 256-byte
  *              aligned (may be NULL when that size is 0).  It holds, between the two kernels of
- *              the linear path, one record of 2112 bytes per row (row scalars and per-segment sums
- *              of w, min(p, q~), max(0, p - q~), p) and one counter per (sequence, trial).
- * Arithmetic of the linear mode: fp32; for N >= 4096 the quotient 1 / (N + p_j) is expanded as
- * (1/N)(1 - x + x^2), x = p_j / N <= 2^-12 (relative truncation below 2^-36), otherwise divided.
+ *              the linear path, one record of 4160 bytes per row (row scalars and per-segment sums
+ *              of w, min(p, q~), max(0, p - q~), p), one counter per (sequence, trial), and 64
+ *              bytes per (row, CTA sharing the row) through which those CTAs exchange their
+ *              partial soft-max sums.  Its contents need no initialisation.
+ * Arithmetic of the linear mode: fp32.  For N >= 4096 with ascending kept ids, 16-byte aligned
+ * target rows and an even drafter row stride, the quotient 1 / (N + p_j) is expanded in
+ * x = p_j / N <= 2^-12 and terms of relative size x^2 (below 2^-24) are dropped; every other
+ * problem takes the one-CTA-per-row kernel, which divides.
  * ------------------------------------------------------------------------------------------- */
 size_t rdk_sample_workspace_bytes(const rdk_problem* problem, int32_t mode, int32_t trials);
 int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* target,

@@ -428,7 +428,7 @@ static int run_rows(const rdk_problem* pb, int mode, const void* target, const v
     P.positions = pb->positions;
     P.accepted_len = out ? out->accepted_len : nullptr;
     if (mode == RDK_MODE_LINEAR && trials > 0 && !force_generic_kernel()) {
-        e = launch_cluster_linear(P, pb->target_dtype, pb->drafter_dtype, pb->drafter_kind, pb->batch, ws, ws_bytes, s);
+        e = launch_stream_linear(P, pb->target_dtype, pb->drafter_dtype, pb->drafter_kind, pb->batch, ws, ws_bytes, s);
         if (e == cudaSuccess) return RDK_OK;          // the draw kernel also wrote accepted_len
     }
     if (e == cudaErrorNotSupported)
@@ -465,7 +465,7 @@ extern "C" size_t rdk_sample_workspace_bytes(const rdk_problem* problem, int32_t
     if (!problem || mode != RDK_MODE_LINEAR || trials < 1 || problem->batch < 1 || problem->positions < 1) return 0;
     const long long rows = (long long)problem->batch * problem->positions;
     if (rows > 0x7fffffffLL) return 0;
-    return cluster_workspace_bytes((int)rows, problem->batch, trials);
+    return stream_workspace_bytes((int)rows, problem->batch, trials);
 }
 
 extern "C" int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* target,

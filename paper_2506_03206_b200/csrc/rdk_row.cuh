@@ -1,4 +1,4 @@
-// Declarations shared by the row kernels (generic one-CTA-per-row kernel and the cluster kernel).
+// Declarations shared by the row kernels (generic one-CTA-per-row kernel and the streaming kernels).
 #pragma once
 
 #include <math.h>
@@ -18,7 +18,7 @@ struct RowParams {
     float* alpha; float* theta; float* S; float* residual_mass; float* qtilde;
     int32_t* status_word;
     int num_tiles;
-    // cluster path only
+    // streaming path only
     int positions;
     int32_t* accepted_len;
     float* rec;            // per-row records in the workspace
@@ -120,7 +120,7 @@ __device__ __forceinline__ int pick_in_segment(const float (&x)[kVec], float rem
 
 // Launches the streaming kernels for the linear path when the problem qualifies; returns
 // cudaErrorNotSupported (and launches nothing) when the generic kernel has to be used.
-cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s);
-size_t cluster_workspace_bytes(int rows, int batch, int trials);
+cudaError_t launch_stream_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s);
+size_t stream_workspace_bytes(int rows, int batch, int trials);
 
 }  // namespace rdk

@@ -963,7 +963,7 @@ static cudaError_t launch_kind_s(const RowParams& P, int kind, const StreamGeo& 
 static size_t ws_off_counters(int rows) { return idx_align((size_t)rows * kRecFloats * sizeof(float)); }
 static size_t ws_off_xrec(int rows, int batch, int trials) { return ws_off_counters(rows) + idx_align((size_t)batch * trials * sizeof(int32_t)); }
 
-size_t cluster_workspace_bytes(int rows, int batch, int trials) {
+size_t stream_workspace_bytes(int rows, int batch, int trials) {
     return ws_off_xrec(rows, batch, trials) + idx_align((size_t)rows * kMaxGroup * kXrecBytes);
 }
 
@@ -976,14 +976,14 @@ static uint32_t next_tag() {
     return t ? t : 0x9E3779B9u;
 }
 
-cudaError_t launch_cluster_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s) {
+cudaError_t launch_stream_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s) {
     const size_t es = tz == RDK_F32 ? 4 : 2, ys = ty == RDK_F32 ? 4 : 2;
     if (P.N < kMinStreamN || P.qtilde || P.rows <= 0 || P.trials <= 0 || !ws) return cudaErrorNotSupported;
     // rows of the target start on 16-byte boundaries; drafter values are read in aligned pairs
     if ((reinterpret_cast<uintptr_t>(P.target) & 15u) || ((P.target_stride * (long long)es) & 15)) return cudaErrorNotSupported;
     if ((reinterpret_cast<uintptr_t>(P.drafter) & 15u) || (P.drafter_stride & 1)) return cudaErrorNotSupported;
     if ((long long)P.rows * P.trials > 0x7fffffffLL) return cudaErrorNotSupported;
-    if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < cluster_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
+    if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < stream_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
     // ascending, valid kept ids only, as recorded when the index was built (kernel 1 re-checks the header)
     if (index_order(P.header) != 1) return cudaErrorNotSupported;
     StreamGeo g;

@@ -150,8 +150,8 @@ def test_identical_distributions_fall_back_to_p_for_the_residual():
     assert torch.allclose(out["alpha"].cpu(), torch.ones(2), atol=1e-6)
 
 
-def test_cluster_of_four_and_two():
-    # 40000 bf16 logits -> four CTAs per row; 12000 fp32 logits -> two
+def test_groups_of_three_and_two_ctas():
+    # 40000 bf16 logits -> three CTAs share a row; 12000 fp32 logits -> two
     cfg = W.tiny_config(N=40000, n=9000, rows=5, dtype="bf16", trials=4, kept_rule="zipf", zipf_bias=True,
                         rho=0.7, seed=41)
     _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
@@ -160,19 +160,19 @@ def test_cluster_of_four_and_two():
 
 
 def test_kept_ids_crowded_into_one_slice():
-    # every kept id lies in the first part of the vocabulary: one CTA's kept-token cache overflows
-    # and the rest of its kept tokens take the uncached route
+    # every kept id lies in the first part of the vocabulary: the kept-token caches of the first warps
+    # overflow and the rest of their kept tokens take the uncached route
     cfg = W.tiny_config(N=70000, n=6000, rows=4, dtype="bf16", trials=8, rho=0.8, seed=43)
     inp = W.make_inputs(cfg)
     ids = torch.arange(cfg.n, dtype=torch.int32) + 100
     _run_linear(cfg, inp, kept_override=ids, check_qtilde=False).assert_ok()
-    # the same ids in a scrambled order (rank -> drafter index table in use)
+    # the same ids in a scrambled order (rank -> drafter index table in use: generic row kernel)
     g = torch.Generator().manual_seed(4)
     _run_linear(cfg, inp, kept_override=ids[torch.randperm(cfg.n, generator=g)], check_qtilde=False).assert_ok()
 
 
-def test_cluster_kernel_agrees_with_generic_kernel_probs_and_full_vocab():
-    # n = N (nothing pruned) and a probability drafter through the cluster kernel
+def test_stream_kernel_probs_and_full_vocab():
+    # n = N (nothing pruned) and a probability drafter through the streaming kernels
     cfg = W.tiny_config(N=8192, n=8192, rows=3, dtype="bf16", trials=8, rho=0.9, seed=44)
     _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
     cfg = W.tiny_config(N=20000, n=4000, rows=3, dtype="bf16", trials=8, drafter_kind="probs", rho=0.8, seed=45)
