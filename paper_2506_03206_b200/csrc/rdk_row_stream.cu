@@ -39,7 +39,6 @@ constexpr int kMaxGroup = 16;            // CTAs that share a row
 constexpr int kMaxSeg = kMaxGroup * kSW; // 256, matches kRecFloats
 constexpr int kMinStreamN = 4096;
 constexpr unsigned kSpinLimit = 1u << 20;
-constexpr unsigned kSuspendHint = 20000;  // time a waiting thread may stay suspended per try, in ns
 constexpr int kDT = 256;                 // threads per CTA of kernel 2: 4 warps for the draft, 4 for the residual
 constexpr int kGW = kDT / 64;            // warps per group of kernel 2
 constexpr int kMaxChunks = 128;          // 256-token chunks per segment
@@ -190,15 +189,21 @@ template <> __device__ __forceinline__ void exp_sum_vec<float>(uint4 q, float2 s
     Ea = fadd2(Ea, e0); Eb = fadd2(Eb, e1);
 }
 
+// Wait for the phase of `bar` with the given parity.  BACKOFF > 0: sleep that many nanoseconds after a
+// failed try (the service warps, which are nearly always early, must not eat issue slots while waiting).
+template <int BACKOFF = 0>
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* fail) {
     unsigned spins = 0;
     uint32_t done = 0;
     while (!done) {
-        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
-                     : "=r"(done) : "r"(bar), "r"(parity), "r"(kSuspendHint) : "memory");
-        if (!done && (++spins > kSpinLimit || ((spins & 1023u) == 0 && *reinterpret_cast<volatile int*>(fail)))) {
-            atomicExch(fail, 1);      // give up: the host reads RDK_ERR_TIMEOUT
-            break;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (!done) {
+            if (++spins > kSpinLimit || ((spins & 1023u) == 0 && *reinterpret_cast<volatile int*>(fail))) {
+                atomicExch(fail, 1);      // give up: the host reads RDK_ERR_TIMEOUT
+                break;
+            }
+            if (BACKOFF > 0) __nanosleep(BACKOFF);
         }
     }
 }
@@ -548,7 +553,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         auto finish_row = [&](int itf) {       // lane w < 16: segment sums of warp w
             const int pf = itf & 1;
             const long long row = grp + (long long)itf * g.G;
-            mbar_wait(smem_u32(&bbar[pf]), (uint32_t)((itf >> 1) & 1), &fail);
+            mbar_wait<100>(smem_u32(&bbar[pf]), (uint32_t)((itf >> 1) & 1), &fail);
             if (lane < kSW) {
                 const float ak = akv[pf][lane];
                 // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
@@ -564,7 +569,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             const int par = it & 1;
             const uint32_t ph = (uint32_t)((it >> 1) & 1);
             const long long row = grp + (long long)it * g.G;
-            mbar_wait(smem_u32(&abar[par]), ph, &fail);
+            mbar_wait<100>(smem_u32(&abar[par]), ph, &fail);
             float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY, K1 = 0.f;
             if (lane < kSW) {
                 const volatile float* wr = &wrec[par][lane][0];
@@ -637,7 +642,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         uint32_t eph = 1, st_a = dsm_a, fb = full_a, eb = empty_a;    // a fresh stage counts as released
         unsigned char* st_p = dsm;
         for (int it = 0; it < rows_g; ++it) {
-            mbar_wait(eb, eph, &fail);
+            mbar_wait<500>(eb, eph, &fail);
             // the few elements a 16-byte copy cannot cover go by plain stores: a slice that ends inside a
             // vector, and the very end of the drafter buffer
             const uintptr_t b0 = reinterpret_cast<uintptr_t>(ny), b1 = b0 + kbytes;
