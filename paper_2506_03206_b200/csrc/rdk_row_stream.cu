@@ -12,8 +12,8 @@
 //                        and publishes it in global memory as five 64-bit words, each a value paired
 //                        with a per-call tag (so every word validates itself and no fence is needed);
 //                        one warp per CTA later polls the C records of the row.
-//   second visit B(row): runs after A(next row), so the exchange latency is hidden; it revisits the
-//                        cached pairs for sum min(p, q~) and writes the segment's sums.
+//   second visit B(row): runs two rows later (after A(row + 2)), so the exchange of a row is off every
+//                        warp's critical path; it revisits the cached pairs for sum min(p, q~).
 // Kernel 2 (rdk_draw_kernel): one CTA per (row, trial) turns the record into draws: it locates the
 // segment by prefix sums, re-reads that one segment (usually still in L2), picks the token, runs
 // the rejection test and the residual draw, and counts the accepted prefix of each sequence.
@@ -42,6 +42,8 @@ constexpr unsigned kSpinLimit = 1u << 20;
 constexpr int kDT = 256;                 // threads per CTA of kernel 2: 4 warps for the draft, 4 for the residual
 constexpr int kGW = kDT / 64;            // warps per group of kernel 2
 constexpr int kMaxChunks = 128;          // 256-token chunks per segment
+constexpr int kDefer = 2;                // rows between a row's first and second visit
+constexpr int kNB = kDefer + 1;          // rows whose records and caches are alive at once
 constexpr int kXrecBytes = 64;           // one published CTA record: five (value, tag) words, padded
 
 // record layout (floats): 16 scalars, then 4 per segment
@@ -288,13 +290,14 @@ template <typename TZ, typename TY, int KIND, int NIT>
 __global__ void __launch_bounds__(kSThreads, 1)
 rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     extern __shared__ __align__(128) unsigned char dsm[];
-    __shared__ __align__(16) float wrec[2][kSW][8];   // [row parity][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), max z, max y
-    __shared__ __align__(16) float scal[2][8];        // [row parity]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta
-    __shared__ __align__(8) float2 fzy[2][kSW];       // [row parity][warp]: factors that turn the warp's cached e_z, e_y into p, q'
-    __shared__ float akv[2][kSW];                     // [row parity][warp]: sum of min(p, q~) over the warp's kept tokens
-    __shared__ __align__(8) unsigned long long abar[2];   // [row parity]: the 16 warp records of the row are in wrec[]
-    __shared__ __align__(8) unsigned long long rbar[2];   // [row parity]: scal[] and fzy[] of the row are set
-    __shared__ __align__(8) unsigned long long bbar[2];   // [row parity]: akv[] of the row is set
+    __shared__ __align__(16) float wrec[kNB][kSW][8];   // [row mod kNB][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), max z, max y
+    __shared__ __align__(16) float scal[kNB][8];        // [row mod kNB]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta
+    __shared__ __align__(8) float2 fzy[kNB][kSW];       // [row mod kNB][warp]: factors that turn the warp's cached e_z, e_y into p, q'
+    __shared__ float akv[kNB][kSW];                     // [row mod kNB][warp]: sum of min(p, q~) over the warp's kept tokens
+    __shared__ __align__(8) unsigned long long abar[kNB];   // [row mod kNB]: the 16 warp records of the row are in wrec[]
+    __shared__ __align__(8) unsigned long long rbar[kNB];   // [row mod kNB]: scal[] and fzy[] of the row are set
+    __shared__ __align__(8) unsigned long long bbar[kNB];   // [row mod kNB]: akv[] of the row is set
+    __shared__ __align__(16) float pend[4][kSW][8];     // exchange warp only, [row mod 4][warp]: the warp's sums, its factors, theta
     __shared__ int fail;
 
     const int tid = threadIdx.x, lane = tid & 31;
@@ -322,14 +325,14 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     const uint32_t zslice = (uint32_t)kSW * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
     const uint32_t stage = zslice + 16u + (uint32_t)kSW * (uint32_t)g.ystage;
     const uint32_t off_cache = (uint32_t)g.NS * stage;
-    const uint32_t off_goff = off_cache + (uint32_t)kSW * 2u * (uint32_t)g.ycap * 8u;
+    const uint32_t off_goff = off_cache + (uint32_t)kSW * (uint32_t)kNB * (uint32_t)g.ycap * 8u;
     const uint32_t off_bar = off_goff + (uint32_t)kSW * (uint32_t)g.ycap * 2u;
     const uint32_t dsm_a = smem_u32(dsm);
     const uint32_t full_a = dsm_a + off_bar, empty_a = full_a + 8u * (uint32_t)g.NS;
 
     if (tid == 0) {
         fail = 0;
-        for (int k = 0; k < 2; ++k) {
+        for (int k = 0; k < kNB; ++k) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&abar[k])), "r"(kSW));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&rbar[k])));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bbar[k])), "r"(kSW));
@@ -386,7 +389,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
         const uint32_t yw_off = zslice + 16u + (uint32_t)warp * (uint32_t)g.ystage;
         const uint32_t csz = (uint32_t)g.ycap * 8u;
-        const uint32_t cb0 = dsm_a + off_cache + (uint32_t)warp * 2u * csz + (uint32_t)lane * 16u;
+        const uint32_t cb0 = dsm_a + off_cache + (uint32_t)warp * (uint32_t)kNB * csz + (uint32_t)lane * 16u;
         const uint32_t gl = dsm_a + off_goff + (uint32_t)warp * (uint32_t)g.ycap * 2u + (uint32_t)lane * 4u;
         // this lane's slots of the pair grid that hold no kept token of the segment (slot 0 when it belongs
         // to the previous segment, and the tail of the last step), as element indices, -1 = none
@@ -398,8 +401,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
 
         // ---- second visit of local row `itb`: sum of min(p, q~) over the cached kept tokens -----------
         auto second_visit = [&](int itb) {
-            const int par = itb & 1;
-            mbar_wait(smem_u32(&rbar[par]), (uint32_t)((itb >> 1) & 1), &fail);
+            const int par = itb % kNB;
+            mbar_wait(smem_u32(&rbar[par]), (uint32_t)((itb / kNB) & 1), &fail);
             const float theta = scal[par][4];
             const float2 f = fzy[par][warp];                  // p = f.x e_z,  q' = f.y e_y
             // q~ = q' + x (theta - q'),  x = p / N
@@ -442,8 +445,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         int s = 0;
         uint32_t sph = 0, st_a = dsm_a, fb = full_a, eb = empty_a;
         unsigned char* st_p = dsm;
+        int par = 0;                                     // it mod kNB
         for (int it = 0; it < rows_g; ++it) {
-            const int par = it & 1;
             const uint32_t zs_a = st_a + zw_off;
             const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(cy) & 15u);      // slot 0 sits this many bytes into the warp's region
             const uint32_t ys_a = st_a + yw_off + shb + (uint32_t)lane * 2u * (uint32_t)sizeof(TY);   // this lane's pair of step 0
@@ -534,95 +537,114 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(eb) : "memory");
             }
 
-            if (it > 0) second_visit(it - 1);
+            if (it >= kDefer) second_visit(it - kDefer);
+            if (++par == kNB) par = 0;
             cy += ystep;
             st_a += stage; st_p += stage; fb += 8u; eb += 8u;
             if (++s == g.NS) { s = 0; sph ^= 1u; st_a = dsm_a; st_p = dsm; fb = full_a; eb = empty_a; }
         }
-        if (rows_g > 0) second_visit(rows_g - 1);
+        for (int itb = max(0, rows_g - kDefer); itb < rows_g; ++itb) second_visit(itb);
     } else if (warp == kSW) {
         // ================================ exchange warp =================================================
-        // per row: fold the CTA's 16 warp records into one and publish it; collect the C records of the
-        // row; leave the row scalars and every warp's factors in shared memory for the second visits;
-        // and turn the previous row's second-visit sums into the per-segment sums the draw kernel reads
-        // lane w < 16 keeps warp w's sums and factors of the row whose second visit is pending in
-        // registers (the shared copies are overwritten two rows on, possibly before that visit ends)
-        float4 w0 = make_float4(0.f, 0.f, 0.f, 0.f);
-        float2 f = make_float2(0.f, 0.f);
-        float theta = 0.f;
-        auto finish_row = [&](int itf) {       // lane w < 16: segment sums of warp w
-            const int pf = itf & 1;
+        // A software pipeline over the rows, so that no global-memory round trip sits between two rows:
+        //   step it     : fold the CTA's 16 warp records of row it into one and publish it;
+        //   step it + 1 : collect the C records of row it (their loads are issued before this step waits
+        //                 for the streaming warps), leave the row scalars and every warp's factors in
+        //                 shared memory for the second visits;
+        //   step it + 3 : the second visits of row it are over: write its per-segment sums.
+        // Lane w < 16 looks after warp w; what a later step needs of a row is parked in pend[row mod 4].
+        auto finish_row = [&](int itf) {
+            const int pf = itf % kNB;
             const long long row = grp + (long long)itf * g.G;
-            mbar_wait<100>(smem_u32(&bbar[pf]), (uint32_t)((itf >> 1) & 1), &fail);
+            mbar_wait<100>(smem_u32(&bbar[pf]), (uint32_t)((itf / kNB) & 1), &fail);
             if (lane < kSW) {
-                const float ak = akv[pf][lane];
+                const float4 w0 = *reinterpret_cast<const float4*>(&pend[itf & 3][lane][0]);
+                const float4 f4 = *reinterpret_cast<const float4*>(&pend[itf & 3][lane][4]);     // fz, fy, theta
+                const float theta = f4.z, ak = akv[pf][lane];
                 // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
-                const float segP = w0.x * f.x;
-                const float xs = f.x * inv_n;
+                const float segP = w0.x * f4.x;
+                const float xs = f4.x * inv_n;
                 const float oov = theta * xs * fmaxf(0.f, w0.x - w0.y);
-                const float Kw = f.y * w0.z - f.y * xs * w0.w + theta * xs * w0.y;
+                const float Kw = f4.y * w0.z - f4.y * xs * w0.w + theta * xs * w0.y;
                 const float a_s = oov + ak;
                 reinterpret_cast<float4*>(P.rec + row * kRecFloats + 16)[seg] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP - a_s), segP);
             }
         };
-        for (int it = 0; it < rows_g; ++it) {
-            const int par = it & 1;
-            const uint32_t ph = (uint32_t)((it >> 1) & 1);
-            const long long row = grp + (long long)it * g.G;
-            mbar_wait<100>(smem_u32(&abar[par]), ph, &fail);
-            float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY, K1 = 0.f;
-            if (lane < kSW) {
-                const volatile float* wr = &wrec[par][lane][0];
-                E1 = wr[0]; K1 = wr[1]; Zq = wr[2]; th = wr[3]; m = wr[4]; my = wr[5];
-            }
-            const float4 w_now = make_float4(E1, K1, Zq, th);
-            const float m_w = m, my_w = my;
-            combine_records(E1, Zq, th, m, my, lane);
-            if (lane == 0) {
-                unsigned char* xr = P.xrec + ((size_t)row * g.C + crank) * kXrecBytes;
-                st_tagged(xr, E1, g.tag); st_tagged(xr + 8, Zq, g.tag); st_tagged(xr + 16, th, g.tag);
-                st_tagged(xr + 24, m, g.tag); st_tagged(xr + 32, my, g.tag);
-            }
-            if (it > 0) finish_row(it - 1);
-            E1 = 0.f; Zq = 0.f; th = 0.f; m = -INFINITY; my = -INFINITY;
-            if (lane < g.C) {
-                const unsigned char* xr = P.xrec + ((size_t)row * g.C + lane) * kXrecBytes;
-                unsigned long long w[5];
-                unsigned spins = 0;
-                for (;;) {
-                    bool ok = true;
+        for (int it = 0; it < rows_g + 3; ++it) {
+            // records of row it - 1: start the loads now
+            const int itc = it - 1;
+            const bool collect = itc >= 0 && itc < rows_g;
+            const long long rowc = grp + (long long)itc * g.G;
+            unsigned long long xw[5] = {0ull, 0ull, 0ull, 0ull, 0ull};
+            if (collect && lane < g.C) {
+                const unsigned char* xr = P.xrec + ((size_t)rowc * g.C + lane) * kXrecBytes;
 #pragma unroll
-                    for (int k = 0; k < 5; ++k) w[k] = ld_tagged(xr + 8 * k);
-#pragma unroll
-                    for (int k = 0; k < 5; ++k) ok = ok && (uint32_t)(w[k] >> 32) == g.tag;
-                    if (ok) break;
-                    if (++spins > kSpinLimit || ld_volatile_s32(&fail)) { atomicExch(&fail, 1); break; }
+                for (int k = 0; k < 5; ++k) xw[k] = ld_tagged(xr + 8 * k);
+            }
+            if (it - 3 >= 0 && it - 3 < rows_g) finish_row(it - 3);
+            if (it < rows_g) {
+                // fold and publish row it
+                const int par = it % kNB;
+                const long long row = grp + (long long)it * g.G;
+                mbar_wait<100>(smem_u32(&abar[par]), (uint32_t)((it / kNB) & 1), &fail);
+                float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY, K1 = 0.f;
+                if (lane < kSW) {
+                    const volatile float* wr = &wrec[par][lane][0];
+                    E1 = wr[0]; K1 = wr[1]; Zq = wr[2]; th = wr[3]; m = wr[4]; my = wr[5];
+                    *reinterpret_cast<float4*>(&pend[it & 3][lane][0]) = make_float4(E1, K1, Zq, th);
+                    *reinterpret_cast<float2*>(&pend[it & 3][lane][4]) = make_float2(m, my);     // the warp's maxima, until the factors replace them
                 }
-                E1 = __uint_as_float((uint32_t)w[0]); Zq = __uint_as_float((uint32_t)w[1]); th = __uint_as_float((uint32_t)w[2]);
-                m = __uint_as_float((uint32_t)w[3]); my = __uint_as_float((uint32_t)w[4]);
-            }
-            combine_records(E1, Zq, th, m, my, lane);
-            const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
-            theta = th * inv_zp * inv_zq;
-            w0 = w_now;
-            f.x = (m_w > -INFINITY ? ex2((m_w - m) * kLog2e) : 0.f) * inv_zp;
-            f.y = (KIND == RDK_LOGITS ? (my_w > -INFINITY ? ex2((my_w - my) * kLog2e) : 0.f) : 1.f) * inv_zq;
-            if (lane < kSW) fzy[par][lane] = f;
-            if (lane == 0) {
-                float* sc = scal[par];
-                sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq; sc[4] = theta;
-                if (crank == 0) {
-                    float* rec = P.rec + row * kRecFloats;
-                    rec[kRecOffg] = sc[0]; rec[kRecInvZp] = inv_zp; rec[kRecYoffg] = sc[2]; rec[kRecInvZq] = inv_zq;
-                    rec[kRecTheta] = theta; rec[kRecInvN] = inv_n; rec[kRecInvS] = 1.f; rec[kRecS] = 1.f;
+                combine_records(E1, Zq, th, m, my, lane);
+                if (lane == 0) {
+                    unsigned char* xr = P.xrec + ((size_t)row * g.C + crank) * kXrecBytes;
+                    st_tagged(xr, E1, g.tag); st_tagged(xr + 8, Zq, g.tag); st_tagged(xr + 16, th, g.tag);
+                    st_tagged(xr + 24, m, g.tag); st_tagged(xr + 32, my, g.tag);
                 }
             }
-            __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[par])) : "memory");
-            if (crank == 0 && P.counters && row % P.positions == 0)
-                for (int t = lane; t < P.trials; t += 32) P.counters[(row / P.positions) * P.trials + t] = 0;
+            if (collect) {
+                const int pc = itc % kNB;
+                float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY;
+                if (lane < g.C) {
+                    const unsigned char* xr = P.xrec + ((size_t)rowc * g.C + lane) * kXrecBytes;
+                    unsigned spins = 0;
+                    for (;;) {
+                        bool ok = true;
+#pragma unroll
+                        for (int k = 0; k < 5; ++k) ok = ok && (uint32_t)(xw[k] >> 32) == g.tag;
+                        if (ok) break;
+                        if (++spins > kSpinLimit || ld_volatile_s32(&fail)) { atomicExch(&fail, 1); break; }
+#pragma unroll
+                        for (int k = 0; k < 5; ++k) xw[k] = ld_tagged(xr + 8 * k);
+                    }
+                    E1 = __uint_as_float((uint32_t)xw[0]); Zq = __uint_as_float((uint32_t)xw[1]); th = __uint_as_float((uint32_t)xw[2]);
+                    m = __uint_as_float((uint32_t)xw[3]); my = __uint_as_float((uint32_t)xw[4]);
+                }
+                combine_records(E1, Zq, th, m, my, lane);
+                const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
+                const float theta = th * inv_zp * inv_zq;
+                if (lane < kSW) {
+                    const float2 mw = *reinterpret_cast<const float2*>(&pend[itc & 3][lane][4]);
+                    float2 f;
+                    f.x = (mw.x > -INFINITY ? ex2((mw.x - m) * kLog2e) : 0.f) * inv_zp;
+                    f.y = (KIND == RDK_LOGITS ? (mw.y > -INFINITY ? ex2((mw.y - my) * kLog2e) : 0.f) : 1.f) * inv_zq;
+                    fzy[pc][lane] = f;
+                    *reinterpret_cast<float4*>(&pend[itc & 3][lane][4]) = make_float4(f.x, f.y, theta, 0.f);
+                }
+                if (lane == 0) {
+                    float* sc = scal[pc];
+                    sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq; sc[4] = theta;
+                    if (crank == 0) {
+                        float* rec = P.rec + rowc * kRecFloats;
+                        rec[kRecOffg] = sc[0]; rec[kRecInvZp] = inv_zp; rec[kRecYoffg] = sc[2]; rec[kRecInvZq] = inv_zq;
+                        rec[kRecTheta] = theta; rec[kRecInvN] = inv_n; rec[kRecInvS] = 1.f; rec[kRecS] = 1.f;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[pc])) : "memory");
+                if (crank == 0 && P.counters && rowc % P.positions == 0)
+                    for (int t = lane; t < P.trials; t += 32) P.counters[(rowc / P.positions) * P.trials + t] = 0;
+            }
         }
-        if (rows_g > 0) finish_row(rows_g - 1);
     } else {
         // ================================ load warp =====================================================
         // per row: one bulk copy of the CTA's slice of the target row and one per warp of the matching
@@ -872,13 +894,13 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
 // ------------------------------------------------------------------------------------------------
 static size_t stream_smem(const StreamGeo& g, size_t es) {
     const size_t stage = (size_t)kSW * g.Lw * es + 16 + (size_t)kSW * g.ystage;
-    return (size_t)g.NS * stage + (size_t)kSW * g.ycap * 18 + (size_t)g.NS * 16;   // + cache (2 x 8 bytes) and offsets (2 bytes) per slot, barriers
+    return (size_t)g.NS * stage + (size_t)kSW * g.ycap * (8 * kNB + 2) + (size_t)g.NS * 16;   // + cache (8 bytes per live row) and offsets (2 bytes) per slot, barriers
 }
 
 // Group size, segment length, stage count and cache capacity for a vocabulary of N tokens with n
 // kept ids; false when the shapes do not fit shared memory.
 static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
-    const size_t budget = 225 * 1024;      // dynamic shared memory a CTA may ask for, less the static part
+    const size_t budget = 222 * 1024;      // dynamic shared memory a CTA may ask for, less the static part
     const int vt = 32 * (int)(16 / es);    // tokens one warp covers with one 16-byte vector per lane
     int C = (N + kSW * 4 * vt - 1) / (kSW * 4 * vt);
     if (C > kMaxGroup) C = kMaxGroup;
