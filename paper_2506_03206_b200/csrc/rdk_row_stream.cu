@@ -34,7 +34,7 @@
 namespace rdk {
 
 constexpr int kSW = 16;                  // warps (= segments) per CTA of kernel 1
-constexpr int kSThreads = (kSW + 2) * 32;   // the streaming warps, the exchange warp and the load warp
+constexpr int kSThreads = (kSW + 3) * 32;   // the streaming warps, the publish warp, the collect warp and the load warp
 constexpr int kMaxGroup = 16;            // CTAs that share a row
 constexpr int kMaxSeg = kMaxGroup * kSW; // 256, matches kRecFloats
 constexpr int kMinStreamN = 4096;
@@ -297,6 +297,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     __shared__ __align__(8) unsigned long long abar[kNB];   // [row mod kNB]: the 16 warp records of the row are in wrec[]
     __shared__ __align__(8) unsigned long long rbar[kNB];   // [row mod kNB]: scal[] and fzy[] of the row are set
     __shared__ __align__(8) unsigned long long bbar[kNB];   // [row mod kNB]: akv[] of the row is set
+    __shared__ __align__(8) unsigned long long pbar[4];     // [row mod 4]: the publish warp has parked the row in pend[]
     __shared__ __align__(16) float pend[4][kSW][8];     // exchange warp only, [row mod 4][warp]: the warp's sums, its factors, theta
     __shared__ int fail;
 
@@ -337,6 +338,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&rbar[k])));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bbar[k])), "r"(kSW));
         }
+        for (int k = 0; k < 4; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&pbar[k])));
         for (int k = 0; k < g.NS; ++k) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_a + 8u * k));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_a + 8u * k), "r"(kSW));
@@ -545,21 +547,17 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         }
         for (int itb = max(0, rows_g - kDefer); itb < rows_g; ++itb) second_visit(itb);
     } else if (warp == kSW) {
-        // ================================ exchange warp =================================================
-        // A software pipeline over the rows, so that no global-memory round trip sits between two rows:
-        //   step it     : fold the CTA's 16 warp records of row it into one and publish it;
-        //   step it + 1 : collect the C records of row it (their loads are issued before this step waits
-        //                 for the streaming warps), leave the row scalars and every warp's factors in
-        //                 shared memory for the second visits;
-        //   step it + 3 : the second visits of row it are over: write its per-segment sums.
-        // Lane w < 16 looks after warp w; what a later step needs of a row is parked in pend[row mod 4].
+        // ================================ publish warp ==================================================
+        // Per row: fold the CTA's 16 warp records into one and publish it in global memory; three rows
+        // later, when the second visits of the row are over, write its per-segment sums.  Lane w < 16
+        // looks after warp w; what later steps need of a row is parked in pend[row mod 4].
         auto finish_row = [&](int itf) {
             const int pf = itf % kNB;
             const long long row = grp + (long long)itf * g.G;
             mbar_wait<100>(smem_u32(&bbar[pf]), (uint32_t)((itf / kNB) & 1), &fail);
             if (lane < kSW) {
                 const float4 w0 = *reinterpret_cast<const float4*>(&pend[itf & 3][lane][0]);
-                const float4 f4 = *reinterpret_cast<const float4*>(&pend[itf & 3][lane][4]);     // fz, fy, theta
+                const float4 f4 = *reinterpret_cast<const float4*>(&pend[itf & 3][lane][4]);     // fz, fy, theta (from the collect warp)
                 const float theta = f4.z, ak = akv[pf][lane];
                 // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
                 const float segP = w0.x * f4.x;
@@ -571,19 +569,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             }
         };
         for (int it = 0; it < rows_g + 3; ++it) {
-            // records of row it - 1: start the loads now
-            const int itc = it - 1;
-            const bool collect = itc >= 0 && itc < rows_g;
-            const long long rowc = grp + (long long)itc * g.G;
-            unsigned long long xw[5] = {0ull, 0ull, 0ull, 0ull, 0ull};
-            if (collect && lane < g.C) {
-                const unsigned char* xr = P.xrec + ((size_t)rowc * g.C + lane) * kXrecBytes;
-#pragma unroll
-                for (int k = 0; k < 5; ++k) xw[k] = ld_tagged(xr + 8 * k);
-            }
-            if (it - 3 >= 0 && it - 3 < rows_g) finish_row(it - 3);
             if (it < rows_g) {
-                // fold and publish row it
                 const int par = it % kNB;
                 const long long row = grp + (long long)it * g.G;
                 mbar_wait<100>(smem_u32(&abar[par]), (uint32_t)((it / kNB) & 1), &fail);
@@ -599,51 +585,60 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                     unsigned char* xr = P.xrec + ((size_t)row * g.C + crank) * kXrecBytes;
                     st_tagged(xr, E1, g.tag); st_tagged(xr + 8, Zq, g.tag); st_tagged(xr + 16, th, g.tag);
                     st_tagged(xr + 24, m, g.tag); st_tagged(xr + 32, my, g.tag);
+                    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&pbar[it & 3])) : "memory");
                 }
             }
-            if (collect) {
-                const int pc = itc % kNB;
-                float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY;
-                if (lane < g.C) {
-                    const unsigned char* xr = P.xrec + ((size_t)rowc * g.C + lane) * kXrecBytes;
-                    unsigned spins = 0;
-                    for (;;) {
-                        bool ok = true;
+            if (it - 3 >= 0) finish_row(it - 3);
+        }
+    } else if (warp == kSW + 1) {
+        // ================================ collect warp ==================================================
+        // Per row: gather the C records of the row from global memory, leave the row scalars and every
+        // warp's factors in shared memory for the second visits.
+        for (int it = 0; it < rows_g; ++it) {
+            const int pc = it % kNB;
+            const long long row = grp + (long long)it * g.G;
+            float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY;
+            if (lane < g.C) {
+                const unsigned char* xr = P.xrec + ((size_t)row * g.C + lane) * kXrecBytes;
+                unsigned long long w[5];
+                unsigned spins = 0;
+                for (;;) {
+                    bool ok = true;
 #pragma unroll
-                        for (int k = 0; k < 5; ++k) ok = ok && (uint32_t)(xw[k] >> 32) == g.tag;
-                        if (ok) break;
-                        if (++spins > kSpinLimit || ld_volatile_s32(&fail)) { atomicExch(&fail, 1); break; }
+                    for (int k = 0; k < 5; ++k) w[k] = ld_tagged(xr + 8 * k);
 #pragma unroll
-                        for (int k = 0; k < 5; ++k) xw[k] = ld_tagged(xr + 8 * k);
-                    }
-                    E1 = __uint_as_float((uint32_t)xw[0]); Zq = __uint_as_float((uint32_t)xw[1]); th = __uint_as_float((uint32_t)xw[2]);
-                    m = __uint_as_float((uint32_t)xw[3]); my = __uint_as_float((uint32_t)xw[4]);
+                    for (int k = 0; k < 5; ++k) ok = ok && (uint32_t)(w[k] >> 32) == g.tag;
+                    if (ok) break;
+                    if (++spins > kSpinLimit || ld_volatile_s32(&fail)) { atomicExch(&fail, 1); break; }
                 }
-                combine_records(E1, Zq, th, m, my, lane);
-                const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
-                const float theta = th * inv_zp * inv_zq;
-                if (lane < kSW) {
-                    const float2 mw = *reinterpret_cast<const float2*>(&pend[itc & 3][lane][4]);
-                    float2 f;
-                    f.x = (mw.x > -INFINITY ? ex2((mw.x - m) * kLog2e) : 0.f) * inv_zp;
-                    f.y = (KIND == RDK_LOGITS ? (mw.y > -INFINITY ? ex2((mw.y - my) * kLog2e) : 0.f) : 1.f) * inv_zq;
-                    fzy[pc][lane] = f;
-                    *reinterpret_cast<float4*>(&pend[itc & 3][lane][4]) = make_float4(f.x, f.y, theta, 0.f);
-                }
-                if (lane == 0) {
-                    float* sc = scal[pc];
-                    sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq; sc[4] = theta;
-                    if (crank == 0) {
-                        float* rec = P.rec + rowc * kRecFloats;
-                        rec[kRecOffg] = sc[0]; rec[kRecInvZp] = inv_zp; rec[kRecYoffg] = sc[2]; rec[kRecInvZq] = inv_zq;
-                        rec[kRecTheta] = theta; rec[kRecInvN] = inv_n; rec[kRecInvS] = 1.f; rec[kRecS] = 1.f;
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[pc])) : "memory");
-                if (crank == 0 && P.counters && rowc % P.positions == 0)
-                    for (int t = lane; t < P.trials; t += 32) P.counters[(rowc / P.positions) * P.trials + t] = 0;
+                E1 = __uint_as_float((uint32_t)w[0]); Zq = __uint_as_float((uint32_t)w[1]); th = __uint_as_float((uint32_t)w[2]);
+                m = __uint_as_float((uint32_t)w[3]); my = __uint_as_float((uint32_t)w[4]);
             }
+            combine_records(E1, Zq, th, m, my, lane);
+            const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
+            const float theta = th * inv_zp * inv_zq;
+            mbar_wait<100>(smem_u32(&pbar[it & 3]), (uint32_t)((it >> 2) & 1), &fail);     // this CTA's own record of the row is parked
+            if (lane < kSW) {
+                const float2 mw = *reinterpret_cast<const float2*>(&pend[it & 3][lane][4]);
+                float2 f;
+                f.x = (mw.x > -INFINITY ? ex2((mw.x - m) * kLog2e) : 0.f) * inv_zp;
+                f.y = (KIND == RDK_LOGITS ? (mw.y > -INFINITY ? ex2((mw.y - my) * kLog2e) : 0.f) : 1.f) * inv_zq;
+                fzy[pc][lane] = f;
+                *reinterpret_cast<float4*>(&pend[it & 3][lane][4]) = make_float4(f.x, f.y, theta, 0.f);
+            }
+            if (lane == 0) {
+                float* sc = scal[pc];
+                sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq; sc[4] = theta;
+                if (crank == 0) {
+                    float* rec = P.rec + row * kRecFloats;
+                    rec[kRecOffg] = sc[0]; rec[kRecInvZp] = inv_zp; rec[kRecYoffg] = sc[2]; rec[kRecInvZq] = inv_zq;
+                    rec[kRecTheta] = theta; rec[kRecInvN] = inv_n; rec[kRecInvS] = 1.f; rec[kRecS] = 1.f;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[pc])) : "memory");
+            if (crank == 0 && P.counters && row % P.positions == 0)
+                for (int t = lane; t < P.trials; t += 32) P.counters[(row / P.positions) * P.trials + t] = 0;
         }
     } else {
         // ================================ load warp =====================================================
