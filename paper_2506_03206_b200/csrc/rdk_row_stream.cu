@@ -42,8 +42,7 @@ constexpr unsigned kSpinLimit = 1u << 20;
 constexpr int kDT = 256;                 // threads per CTA of kernel 2: 4 warps for the draft, 4 for the residual
 constexpr int kGW = kDT / 64;            // warps per group of kernel 2
 constexpr int kMaxChunks = 128;          // 256-token chunks per segment
-constexpr int kDefer = 2;                // rows between a row's first and second visit
-constexpr int kNB = kDefer + 1;          // rows whose records and caches are alive at once
+constexpr int kMaxNB = 6;                // most rows whose records and caches are alive at once (StreamGeo::NB)
 constexpr int kXrecBytes = 64;           // one published CTA record: five (value, tag) words, padded
 
 // record layout (floats): 16 scalars, then 4 per segment
@@ -56,6 +55,8 @@ struct StreamGeo {
     int Lw;                // tokens per segment: nv vectors of 16 bytes per lane
     int nv;
     int NS;                // stages
+    int NB;                // rows whose records and caches are alive at once: the second visit of a row
+                           // follows its first visit NB - 1 rows later
     int ycap;              // kept-token slots per warp that are staged and cached (multiple of 64)
     int ystage;            // bytes of a warp's drafter region in a stage
     uint32_t tag;          // value that marks a record word as written by this call
@@ -290,15 +291,15 @@ template <typename TZ, typename TY, int KIND, int NIT>
 __global__ void __launch_bounds__(kSThreads, 1)
 rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     extern __shared__ __align__(128) unsigned char dsm[];
-    __shared__ __align__(16) float wrec[kNB][kSW][8];   // [row mod kNB][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), max z, max y
-    __shared__ __align__(16) float scal[kNB][8];        // [row mod kNB]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta
-    __shared__ __align__(8) float2 fzy[kNB][kSW];       // [row mod kNB][warp]: factors that turn the warp's cached e_z, e_y into p, q'
-    __shared__ float akv[kNB][kSW];                     // [row mod kNB][warp]: sum of min(p, q~) over the warp's kept tokens
-    __shared__ __align__(8) unsigned long long abar[kNB];   // [row mod kNB]: the 16 warp records of the row are in wrec[]
-    __shared__ __align__(8) unsigned long long rbar[kNB];   // [row mod kNB]: scal[] and fzy[] of the row are set
-    __shared__ __align__(8) unsigned long long bbar[kNB];   // [row mod kNB]: akv[] of the row is set
-    __shared__ __align__(8) unsigned long long pbar[4];     // [row mod 4]: the publish warp has parked the row in pend[]
-    __shared__ __align__(16) float pend[4][kSW][8];     // exchange warp only, [row mod 4][warp]: the warp's sums, its factors, theta
+    __shared__ __align__(16) float wrec[kMaxNB][kSW][8];   // [row mod NB][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), max z, max y
+    __shared__ __align__(16) float scal[kMaxNB][8];        // [row mod NB]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta
+    __shared__ __align__(8) float2 fzy[kMaxNB][kSW];       // [row mod NB][warp]: factors that turn the warp's cached e_z, e_y into p, q'
+    __shared__ float akv[kMaxNB][kSW];                     // [row mod NB][warp]: sum of min(p, q~) over the warp's kept tokens
+    __shared__ __align__(8) unsigned long long abar[kMaxNB];   // [row mod NB]: the 16 warp records of the row are in wrec[]
+    __shared__ __align__(8) unsigned long long rbar[kMaxNB];   // [row mod NB]: scal[] and fzy[] of the row are set
+    __shared__ __align__(8) unsigned long long bbar[kMaxNB];   // [row mod NB]: akv[] of the row is set
+    __shared__ __align__(8) unsigned long long pbar[8];     // [row mod 8]: the publish warp has parked the row in pend[]
+    __shared__ __align__(16) float pend[8][kSW][8];     // publish and collect warps only, [row mod 8][warp]: the warp's sums, its factors, theta
     __shared__ int fail;
 
     const int tid = threadIdx.x, lane = tid & 31;
@@ -326,19 +327,20 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     const uint32_t zslice = (uint32_t)kSW * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
     const uint32_t stage = zslice + 16u + (uint32_t)kSW * (uint32_t)g.ystage;
     const uint32_t off_cache = (uint32_t)g.NS * stage;
-    const uint32_t off_goff = off_cache + (uint32_t)kSW * (uint32_t)kNB * (uint32_t)g.ycap * 8u;
+    const int nb = g.NB, defer = g.NB - 1;
+    const uint32_t off_goff = off_cache + (uint32_t)kSW * (uint32_t)nb * (uint32_t)g.ycap * 8u;
     const uint32_t off_bar = off_goff + (uint32_t)kSW * (uint32_t)g.ycap * 2u;
     const uint32_t dsm_a = smem_u32(dsm);
     const uint32_t full_a = dsm_a + off_bar, empty_a = full_a + 8u * (uint32_t)g.NS;
 
     if (tid == 0) {
         fail = 0;
-        for (int k = 0; k < kNB; ++k) {
+        for (int k = 0; k < kMaxNB; ++k) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&abar[k])), "r"(kSW));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&rbar[k])));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bbar[k])), "r"(kSW));
         }
-        for (int k = 0; k < 4; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&pbar[k])));
+        for (int k = 0; k < 8; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&pbar[k])));
         for (int k = 0; k < g.NS; ++k) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_a + 8u * k));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_a + 8u * k), "r"(kSW));
@@ -391,7 +393,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
         const uint32_t yw_off = zslice + 16u + (uint32_t)warp * (uint32_t)g.ystage;
         const uint32_t csz = (uint32_t)g.ycap * 8u;
-        const uint32_t cb0 = dsm_a + off_cache + (uint32_t)warp * (uint32_t)kNB * csz + (uint32_t)lane * 16u;
+        const uint32_t cb0 = dsm_a + off_cache + (uint32_t)warp * (uint32_t)nb * csz + (uint32_t)lane * 16u;
         const uint32_t gl = dsm_a + off_goff + (uint32_t)warp * (uint32_t)g.ycap * 2u + (uint32_t)lane * 4u;
         // this lane's slots of the pair grid that hold no kept token of the segment (slot 0 when it belongs
         // to the previous segment, and the tail of the last step), as element indices, -1 = none
@@ -402,9 +404,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         const float2 l2e = splat(kLog2e);
 
         // ---- second visit of local row `itb`: sum of min(p, q~) over the cached kept tokens -----------
-        auto second_visit = [&](int itb) {
-            const int par = itb % kNB;
-            mbar_wait(smem_u32(&rbar[par]), (uint32_t)((itb / kNB) & 1), &fail);
+        auto second_visit = [&](int itb, int par, uint32_t ph) {       // par = itb mod NB, ph = parity of itb / NB
+            mbar_wait(smem_u32(&rbar[par]), ph, &fail);
             const float theta = scal[par][4];
             const float2 f = fzy[par][warp];                  // p = f.x e_z,  q' = f.y e_y
             // q~ = q' + x (theta - q'),  x = p / N
@@ -447,7 +448,9 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         int s = 0;
         uint32_t sph = 0, st_a = dsm_a, fb = full_a, eb = empty_a;
         unsigned char* st_p = dsm;
-        int par = 0;                                     // it mod kNB
+        int par = 0;                                     // it mod NB
+        int bit = 0, bpar = 0;                           // next row to get its second visit, the same mod NB
+        uint32_t bph = 0;
         for (int it = 0; it < rows_g; ++it) {
             const uint32_t zs_a = st_a + zw_off;
             const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(cy) & 15u);      // slot 0 sits this many bytes into the warp's region
@@ -539,25 +542,32 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(eb) : "memory");
             }
 
-            if (it >= kDefer) second_visit(it - kDefer);
-            if (++par == kNB) par = 0;
+            if (it >= defer) {
+                second_visit(bit, bpar, bph);
+                ++bit;
+                if (++bpar == nb) { bpar = 0; bph ^= 1u; }
+            }
+            if (++par == nb) par = 0;
             cy += ystep;
             st_a += stage; st_p += stage; fb += 8u; eb += 8u;
             if (++s == g.NS) { s = 0; sph ^= 1u; st_a = dsm_a; st_p = dsm; fb = full_a; eb = empty_a; }
         }
-        for (int itb = max(0, rows_g - kDefer); itb < rows_g; ++itb) second_visit(itb);
+        for (; bit < rows_g; ++bit) {
+            second_visit(bit, bpar, bph);
+            if (++bpar == nb) { bpar = 0; bph ^= 1u; }
+        }
     } else if (warp == kSW) {
         // ================================ publish warp ==================================================
-        // Per row: fold the CTA's 16 warp records into one and publish it in global memory; three rows
+        // Per row: fold the CTA's 16 warp records into one and publish it in global memory; NB rows
         // later, when the second visits of the row are over, write its per-segment sums.  Lane w < 16
-        // looks after warp w; what later steps need of a row is parked in pend[row mod 4].
+        // looks after warp w; what later steps need of a row is parked in pend[row mod 8].
         auto finish_row = [&](int itf) {
-            const int pf = itf % kNB;
+            const int pf = itf % nb;
             const long long row = grp + (long long)itf * g.G;
-            mbar_wait<100>(smem_u32(&bbar[pf]), (uint32_t)((itf / kNB) & 1), &fail);
+            mbar_wait<100>(smem_u32(&bbar[pf]), (uint32_t)((itf / nb) & 1), &fail);
             if (lane < kSW) {
-                const float4 w0 = *reinterpret_cast<const float4*>(&pend[itf & 3][lane][0]);
-                const float4 f4 = *reinterpret_cast<const float4*>(&pend[itf & 3][lane][4]);     // fz, fy, theta (from the collect warp)
+                const float4 w0 = *reinterpret_cast<const float4*>(&pend[itf & 7][lane][0]);
+                const float4 f4 = *reinterpret_cast<const float4*>(&pend[itf & 7][lane][4]);     // fz, fy, theta (from the collect warp)
                 const float theta = f4.z, ak = akv[pf][lane];
                 // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
                 const float segP = w0.x * f4.x;
@@ -568,34 +578,34 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 reinterpret_cast<float4*>(P.rec + row * kRecFloats + 16)[seg] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP - a_s), segP);
             }
         };
-        for (int it = 0; it < rows_g + 3; ++it) {
+        for (int it = 0; it < rows_g + nb; ++it) {
             if (it < rows_g) {
-                const int par = it % kNB;
+                const int par = it % nb;
                 const long long row = grp + (long long)it * g.G;
-                mbar_wait<100>(smem_u32(&abar[par]), (uint32_t)((it / kNB) & 1), &fail);
+                mbar_wait<100>(smem_u32(&abar[par]), (uint32_t)((it / nb) & 1), &fail);
                 float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY, K1 = 0.f;
                 if (lane < kSW) {
                     const volatile float* wr = &wrec[par][lane][0];
                     E1 = wr[0]; K1 = wr[1]; Zq = wr[2]; th = wr[3]; m = wr[4]; my = wr[5];
-                    *reinterpret_cast<float4*>(&pend[it & 3][lane][0]) = make_float4(E1, K1, Zq, th);
-                    *reinterpret_cast<float2*>(&pend[it & 3][lane][4]) = make_float2(m, my);     // the warp's maxima, until the factors replace them
+                    *reinterpret_cast<float4*>(&pend[it & 7][lane][0]) = make_float4(E1, K1, Zq, th);
+                    *reinterpret_cast<float2*>(&pend[it & 7][lane][4]) = make_float2(m, my);     // the warp's maxima, until the factors replace them
                 }
                 combine_records(E1, Zq, th, m, my, lane);
                 if (lane == 0) {
                     unsigned char* xr = P.xrec + ((size_t)row * g.C + crank) * kXrecBytes;
                     st_tagged(xr, E1, g.tag); st_tagged(xr + 8, Zq, g.tag); st_tagged(xr + 16, th, g.tag);
                     st_tagged(xr + 24, m, g.tag); st_tagged(xr + 32, my, g.tag);
-                    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&pbar[it & 3])) : "memory");
+                    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&pbar[it & 7])) : "memory");
                 }
             }
-            if (it - 3 >= 0) finish_row(it - 3);
+            if (it - nb >= 0) finish_row(it - nb);
         }
     } else if (warp == kSW + 1) {
         // ================================ collect warp ==================================================
         // Per row: gather the C records of the row from global memory, leave the row scalars and every
         // warp's factors in shared memory for the second visits.
         for (int it = 0; it < rows_g; ++it) {
-            const int pc = it % kNB;
+            const int pc = it % nb;
             const long long row = grp + (long long)it * g.G;
             float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY;
             if (lane < g.C) {
@@ -617,14 +627,14 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             combine_records(E1, Zq, th, m, my, lane);
             const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
             const float theta = th * inv_zp * inv_zq;
-            mbar_wait<100>(smem_u32(&pbar[it & 3]), (uint32_t)((it >> 2) & 1), &fail);     // this CTA's own record of the row is parked
+            mbar_wait<100>(smem_u32(&pbar[it & 7]), (uint32_t)((it >> 3) & 1), &fail);     // this CTA's own record of the row is parked
             if (lane < kSW) {
-                const float2 mw = *reinterpret_cast<const float2*>(&pend[it & 3][lane][4]);
+                const float2 mw = *reinterpret_cast<const float2*>(&pend[it & 7][lane][4]);
                 float2 f;
                 f.x = (mw.x > -INFINITY ? ex2((mw.x - m) * kLog2e) : 0.f) * inv_zp;
                 f.y = (KIND == RDK_LOGITS ? (mw.y > -INFINITY ? ex2((mw.y - my) * kLog2e) : 0.f) : 1.f) * inv_zq;
                 fzy[pc][lane] = f;
-                *reinterpret_cast<float4*>(&pend[it & 3][lane][4]) = make_float4(f.x, f.y, theta, 0.f);
+                *reinterpret_cast<float4*>(&pend[it & 7][lane][4]) = make_float4(f.x, f.y, theta, 0.f);
             }
             if (lane == 0) {
                 float* sc = scal[pc];
@@ -889,13 +899,13 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
 // ------------------------------------------------------------------------------------------------
 static size_t stream_smem(const StreamGeo& g, size_t es) {
     const size_t stage = (size_t)kSW * g.Lw * es + 16 + (size_t)kSW * g.ystage;
-    return (size_t)g.NS * stage + (size_t)kSW * g.ycap * (8 * kNB + 2) + (size_t)g.NS * 16;   // + cache (8 bytes per live row) and offsets (2 bytes) per slot, barriers
+    return (size_t)g.NS * stage + (size_t)kSW * g.ycap * (8 * g.NB + 2) + (size_t)g.NS * 16;   // + cache (8 bytes per live row) and offsets (2 bytes) per slot, barriers
 }
 
 // Group size, segment length, stage count and cache capacity for a vocabulary of N tokens with n
 // kept ids; false when the shapes do not fit shared memory.
 static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
-    const size_t budget = 222 * 1024;      // dynamic shared memory a CTA may ask for, less the static part
+    const size_t budget = 218 * 1024;      // dynamic shared memory a CTA may ask for, less the static part (about 9 KB)
     const int vt = 32 * (int)(16 / es);    // tokens one warp covers with one 16-byte vector per lane
     int C = (N + kSW * 4 * vt - 1) / (kSW * 4 * vt);
     if (C > kMaxGroup) C = kMaxGroup;
@@ -908,15 +918,19 @@ static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
     const long long most = (long long)(n < g.Lw ? n : g.Lw) + 1;
     if (cap > most) cap = most;
     cap = (cap + 63) / 64 * 64;
-    for (g.NS = 3; g.NS >= 2; --g.NS) {
-        long long c = cap;
-        while (c >= 64) {
-            g.ycap = (int)c;
-            g.ystage = (int)((((size_t)c + 16) * ys + 15) & ~size_t(15));
-            if (stream_smem(g, es) <= budget) return true;
-            if (g.NS > 2) break;          // first give up a stage, then cache capacity
-            c -= 64;
-        }
+    // The exchange of a row between the CTAs of its group takes about as long as two first visits, so
+    // the second visit should trail by several rows: prefer live rows over stages, then give up cache.
+    static const int pref[][2] = {{5, 2}, {4, 2}, {3, 3}, {3, 2}};     // {NB, NS}
+    for (const auto& pr : pref) {
+        g.NB = pr[0]; g.NS = pr[1];
+        g.ycap = (int)cap;
+        g.ystage = (int)((((size_t)cap + 16) * ys + 15) & ~size_t(15));
+        if (stream_smem(g, es) <= budget) return true;
+    }
+    for (long long c = cap - 64; c >= 64; c -= 64) {
+        g.ycap = (int)c;
+        g.ystage = (int)((((size_t)c + 16) * ys + 15) & ~size_t(15));
+        if (stream_smem(g, es) <= budget) return true;
     }
     return false;
 }
