@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "bd1431533f5a4a8a5dc5c86dc9bdc10a77071a5f8c02ae3865a32b8005f2e12c",
-               "bytes_per_launch": 102922496 + 3479552}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
+NCU_TRAFFIC = {"sources_sha256": "592f9bcaded9b93ff8f5ec7c421aa7075c5000be20635f6a341fc99d66150018",
+               "bytes_per_launch": 102940928 + 4625408}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 
