@@ -39,8 +39,6 @@ constexpr int kMaxGroup = 16;            // CTAs that share a row
 constexpr int kMaxSeg = kMaxGroup * kSW; // 256, matches kRecFloats
 constexpr int kMinStreamN = 4096;
 constexpr unsigned kSpinLimit = 1u << 20;
-constexpr int kDT = 256;                 // threads per CTA of kernel 2: 4 warps for the draft, 4 for the residual
-constexpr int kGW = kDT / 64;            // warps per group of kernel 2
 constexpr int kMaxChunks = 128;          // 256-token chunks per segment
 constexpr int kMaxNB = 6;                // most rows whose records and caches are alive at once (StreamGeo::NB)
 constexpr int kXrecBytes = 64;           // one published CTA record: five (value, tag) words, padded
@@ -757,8 +755,9 @@ __device__ __forceinline__ void draw_x(const DrawCtx& d, int what, int jb, int s
         x[k] = what == kPickW ? w[k] : (what == kPickR ? fmaxf(0.f, p[k] - w[k] * d.c.inv_s) : p[k]);
 }
 
-template <typename TZ, typename TY, int KIND>
-__global__ void __launch_bounds__(kDT)
+// DT threads per CTA: half of the warps work on the draft draw, half on the residual draw.
+template <typename TZ, typename TY, int KIND, int DT>
+__global__ void __launch_bounds__(DT)
 rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
     __shared__ double cdfW[kMaxSeg], cdfR[kMaxSeg], cdfP[kMaxSeg];
     __shared__ float sums[2][kMaxChunks];
@@ -819,6 +818,7 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
 
     // group 0 (first half of the warps): the draft draw from w; group 1: the residual draw, computed
     // alongside (it is only used if the draft is rejected)
+    constexpr int kGW = DT / 64;             // warps per group
     const int g = warp / kGW, wg = warp % kGW;
     const bool from_p = !(R_d > 0.0);                 // p and q~ coincide: the replacement comes from p itself
     const double* cdf = g == 0 ? cdfW : (from_p ? cdfP : cdfR);
@@ -971,9 +971,15 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
     cfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&cfg, kern, P, g);
     if (e != cudaSuccess) return e;
+    // small CTAs when the draws of all rows would not be resident at once with large ones (shorter
+    // tail), large CTAs otherwise (shorter chain per row)
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const bool small_ctas = (long long)P.rows * P.trials > (long long)sms * 8;
     cudaLaunchConfig_t dcfg = {};
     dcfg.gridDim = dim3((unsigned)(P.rows * P.trials), 1, 1);
-    dcfg.blockDim = dim3(kDT, 1, 1);
+    dcfg.blockDim = dim3(small_ctas ? 128 : 256, 1, 1);
     dcfg.dynamicSmemBytes = 0;
     dcfg.stream = s;
     cudaLaunchAttribute dattr[1];
@@ -981,7 +987,8 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
     dattr[0].val.programmaticStreamSerializationAllowed = 1;
     dcfg.attrs = dattr;
     dcfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&dcfg, rdk_draw_kernel<TZ, TY, KIND>, P, g.C * kSW, g.Lw);
+    if (small_ctas) return cudaLaunchKernelEx(&dcfg, rdk_draw_kernel<TZ, TY, KIND, 128>, P, g.C * kSW, g.Lw);
+    return cudaLaunchKernelEx(&dcfg, rdk_draw_kernel<TZ, TY, KIND, 256>, P, g.C * kSW, g.Lw);
 }
 
 template <typename TZ, typename TY, int KIND>
