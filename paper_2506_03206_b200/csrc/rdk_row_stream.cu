@@ -777,29 +777,28 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
     d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
     d.c.inv_s = __ldcg(rec + kRecInvS);
 
-    if (warp == 0) {   // prefix sums over the segments, fp64
-        double cw = 0.0, cr = 0.0, cp = 0.0;
-        float alpha_l = 0.f;
+    if (warp < 3) {   // fp64 prefix sums over the segments: warp 0 those of w, warp 1 of max(0, p - q~), warp 2 of p
+        double* cdf = warp == 0 ? cdfW : (warp == 1 ? cdfR : cdfP);
+        double carry = 0.0;
         for (int base = 0; base < nseg; base += 32) {
             const int s = base + lane;
-            double iw = 0.0, ir = 0.0, ip = 0.0;
+            double x = 0.0;
             if (s < nseg) {
                 const float4 v = __ldcg(reinterpret_cast<const float4*>(rec + 16) + s);
-                iw = (double)v.x; alpha_l += v.y; ir = (double)v.z; ip = (double)v.w;
+                x = (double)(warp == 0 ? v.x : (warp == 1 ? v.z : v.w));
             }
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const double a = __shfl_up_sync(0xffffffffu, iw, o);
-                const double b = __shfl_up_sync(0xffffffffu, ir, o);
-                const double e = __shfl_up_sync(0xffffffffu, ip, o);
-                if (lane >= o) { iw += a; ir += b; ip += e; }
+                const double a = __shfl_up_sync(0xffffffffu, x, o);
+                if (lane >= o) x += a;
             }
-            iw += cw; ir += cr; ip += cp;
-            cw = __shfl_sync(0xffffffffu, iw, 31);
-            cr = __shfl_sync(0xffffffffu, ir, 31);
-            cp = __shfl_sync(0xffffffffu, ip, 31);
-            if (s < nseg) { cdfW[s] = iw; cdfR[s] = ir; cdfP[s] = ip; }
+            x += carry;
+            carry = __shfl_sync(0xffffffffu, x, 31);
+            if (s < nseg) cdf[s] = x;
         }
+    } else if (warp == 3) {   // alpha = sum over the segments of sum min(p, q~)
+        float alpha_l = 0.f;
+        for (int s = lane; s < nseg; s += 32) alpha_l += __ldcg(reinterpret_cast<const float4*>(rec + 16) + s).y;
         alpha_l = warp_sum(alpha_l);
         if (lane == 0) alpha_s = alpha_l;
     }
