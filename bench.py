@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "592f9bcaded9b93ff8f5ec7c421aa7075c5000be20635f6a341fc99d66150018",
-               "bytes_per_launch": 102940928 + 4625408}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
+NCU_TRAFFIC = {"sources_sha256": "6af51d298601141aedfe53612e7b89e65b578828b83873dc4bc11c65ab44c19e",
+               "bytes_per_launch": 102939648 + 3941632}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 
