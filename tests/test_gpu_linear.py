@@ -179,6 +179,41 @@ def test_stream_kernel_probs_and_full_vocab():
     _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
 
 
+def test_many_rows_per_group_every_row_checked():
+    """A group of three CTAs takes some thirty rows in turn: stages, live-row buffers and barrier
+    phases all wrap several times.  Every row is compared with the checker."""
+    cfg = W.tiny_config(N=40000, n=7000, rows=1500, dtype="bf16", trials=1, kept_rule="zipf", zipf_bias=True,
+                        rho=0.8, seed=51)
+    _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
+
+
+def test_few_rows_fewer_than_the_pipeline_depth():
+    # one and two rows: the deferred second visits all happen after the row loop
+    for rows in (1, 2):
+        cfg = W.tiny_config(N=20000, n=3000, rows=rows, dtype="bf16", trials=8, rho=0.6, seed=52 + rows)
+        _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
+
+
+def test_strided_rows_through_the_streaming_kernels():
+    """Rows embedded in wider buffers (target stride a multiple of 8 elements, drafter stride even but
+    not a multiple of 8, so the drafter rows start at varying 16-byte phases)."""
+    rdk = _rdk()
+    B = rdk.binding
+    cfg = W.tiny_config(N=24576, n=5001, rows=40, dtype="bf16", trials=2, kept_rule="zipf", zipf_bias=True,
+                        rho=0.7, seed=57)
+    inp = W.make_inputs(cfg)
+    tw = torch.zeros(cfg.rows, cfg.N + 24, dtype=torch.bfloat16)
+    tw[:, : cfg.N] = inp["target"]
+    dw = torch.zeros(cfg.rows, cfg.n + 5, dtype=torch.bfloat16)
+    dw[:, : cfg.n] = inp["drafter"]
+    idx = rdk.rdk_prepare_ids(inp["kept_ids"].cuda(), cfg.N)
+    out = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, tw.cuda()[:, : cfg.N], dw.cuda()[:, : cfg.n], None,
+                                    inp["uniforms"].cuda(), cfg.batch, cfg.positions)
+    torch.cuda.synchronize()
+    B.check_status_word(out)
+    PU.compare_sampling(inp, out, range(cfg.rows), "linear").assert_ok()
+
+
 @pytest.mark.parametrize("name,nrows", [("C2", 10), ("C3", 8), ("C4", 6)])
 def test_full_size_configs_sampled_rows(name, nrows):
     """Full-size workloads in the launch configuration the benchmark times; the checker recomputes a
