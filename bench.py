@@ -32,7 +32,7 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "6af51d298601141aedfe53612e7b89e65b578828b83873dc4bc11c65ab44c19e",
+NCU_TRAFFIC = {"sources_sha256": "4378ea64417149cb325d86fb2757d469bc59b79e9e2525ec21afc3196b6ad9c4",
                "bytes_per_launch": 102939648 + 3941632}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 

@@ -1,19 +1,24 @@
 // Two-kernel form of the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8) for N >= 4096
 // and kept ids in ascending order.
 //
-// Kernel 1 (rdk_stream_kernel): a persistent grid of G groups of C CTAs, 16 warps each.  Group g
-// takes rows g, g + G, ...; within a row, warp w of CTA c owns the contiguous token range
-// ("segment") s = 16 c + w.  Every warp runs its own pipeline: a ring of NS shared-memory stages
-// filled by TMA bulk copies (its slice of the target logits and the matching contiguous run of
-// drafter values), so a row is read from HBM exactly once and no block-wide barrier exists.
-//   first visit  A(row): maxima, sum of e = exp(z - max) over the segment, and over the segment's
-//                        kept tokens sum e_z, sum e_y, sum e_z e_y; (e_z, e_y) pairs are cached.
-//   exchange           : the last warp of a CTA to finish A(row) folds the 16 warp records into one
-//                        and publishes it in global memory as five 64-bit words, each a value paired
-//                        with a per-call tag (so every word validates itself and no fence is needed);
-//                        one warp per CTA later polls the C records of the row.
-//   second visit B(row): runs two rows later (after A(row + 2)), so the exchange of a row is off every
-//                        warp's critical path; it revisits the cached pairs for sum min(p, q~).
+// Kernel 1 (rdk_stream_kernel): a persistent grid of G groups of C CTAs, one CTA per SM.  Group g
+// takes rows g, g + G, ...; within a row, streaming warp w of CTA c owns the contiguous token range
+// ("segment") s = 16 c + w.  A CTA has 19 warps and no block-wide barrier in its row loop:
+//   load warp      : per row, one bulk copy (TMA) of the CTA's slice of the target logits and one per
+//                    streaming warp of the matching contiguous run of drafter values, into a ring of
+//                    NS shared-memory stages, so a row is read from HBM exactly once.
+//   16 streaming warps, first visit A(row): maxima, sum of e = exp(z - max) over the segment, and
+//                    over the segment's kept tokens sum e_z, sum e_y, sum e_z e_y; the (e_z, e_y)
+//                    pairs are cached.  Second visit B(row), NB - 1 rows later: sum min(p, q~) over
+//                    the cached pairs, when the row's scalars are known.
+//   publish warp   : folds the CTA's 16 warp records of a row into one and publishes it in global
+//                    memory as five 64-bit words, each a value paired with a per-call tag (so every
+//                    word validates itself and no fence is needed); NB rows later, writes the row's
+//                    per-segment sums.
+//   collect warp   : polls the C records of a row and leaves the row scalars and every warp's scale
+//                    factors in shared memory for the second visits.
+// The exchange of a row costs about two first visits of latency; with the second visit trailing by
+// NB - 1 rows and the exchange in warps of its own, it is off the streaming warps' critical path.
 // Kernel 2 (rdk_draw_kernel): one CTA per (row, trial) turns the record into draws: it locates the
 // segment by prefix sums, re-reads that one segment (usually still in L2), picks the token, runs
 // the rejection test and the residual draw, and counts the accepted prefix of each sequence.
