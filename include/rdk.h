@@ -222,6 +222,31 @@ int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* 
                           void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * rdk_stream_geometry -- host-only query (no CUDA call): how the streaming kernels of the linear
+ * mode would lay a problem of N target tokens and n kept ids out, or supported = 0 when such a
+ * problem takes the one-CTA-per-row kernel (N < 4096, or shapes beyond shared memory; unsorted
+ * or invalid kept ids and unaligned rows also do, but are not known here).  A row is shared by
+ * ctas_per_row CTAs of warps_per_cta streaming warps, each owning segment_tokens consecutive
+ * tokens (Eq. "rdk-taylor" is evaluated per segment; ctas_per_row * warps_per_cta segments cover
+ * the vocabulary); stages = depth of the shared-memory ring; live_rows - 1 = rows by which the
+ * second visit of a row trails its first.  Returns RDK_OK, or RDK_ERR_INVALID_ARG.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct rdk_stream_geometry_t {
+    int32_t supported;
+    int32_t ctas_per_row;
+    int32_t warps_per_cta;
+    int32_t segment_tokens;
+    int32_t stages;
+    int32_t live_rows;
+    int32_t cached_slots_per_warp;
+    int32_t reserved;
+    int64_t dynamic_shared_bytes;
+} rdk_stream_geometry_t;
+int rdk_stream_geometry(int32_t N, int32_t n, int32_t target_dtype, int32_t drafter_dtype,
+                        rdk_stream_geometry_t* out);
+
+
+/* ---------------------------------------------------------------------------------------------
  * rdk_emit_sequences -- Algorithm 4 steps 7-9: what each sequence emits after verification.  For
  * sequence b and trial t, with j = number of leading accepted positions:
  *   seq_tokens[b, t, 0..j) = the accepted drafts d_1..d_j,

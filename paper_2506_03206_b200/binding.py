@@ -30,7 +30,7 @@ EXPORTS = [
     "rdk_build_affinity_workspace_bytes", "rdk_build_affinity", "rdk_exact_workspace_bytes",
     "rdk_redistribute_exact", "rdk_redistribute_exact_static", "rdk_redistribute_linear",
     "rdk_sample_workspace_bytes", "rdk_sample_and_verify", "rdk_emit_sequences",
-    "rdk_sample_and_verify_host",
+    "rdk_sample_and_verify_host", "rdk_stream_geometry",
 ]
 
 
@@ -49,6 +49,12 @@ class rdk_problem(C.Structure):
 
 class rdk_affinity(C.Structure):
     _fields_ = [("data", C.c_void_p), ("layout", C.c_int32), ("reserved", C.c_int32), ("ld", C.c_int64)]
+
+
+class rdk_stream_geometry_t(C.Structure):
+    _fields_ = [("supported", C.c_int32), ("ctas_per_row", C.c_int32), ("warps_per_cta", C.c_int32),
+                ("segment_tokens", C.c_int32), ("stages", C.c_int32), ("live_rows", C.c_int32),
+                ("cached_slots_per_warp", C.c_int32), ("reserved", C.c_int32), ("dynamic_shared_bytes", C.c_int64)]
 
 
 class rdk_outputs(C.Structure):
@@ -354,3 +360,13 @@ def check_status_word(out: Dict[str, torch.Tensor], where: str = "kernel") -> No
     code = int(out["status_word"].item())
     if code != 0:
         raise RdkError(code, where, lib().rdk_status_string(code).decode())
+
+
+def rdk_stream_geometry(N: int, n: int, target_dtype: int = RDK_BF16, drafter_dtype: int = RDK_BF16) -> Dict[str, int]:
+    """How the streaming kernels of the linear mode would lay out a problem (host-only query)."""
+    L = lib()
+    L.rdk_stream_geometry.restype = C.c_int
+    L.rdk_stream_geometry.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(rdk_stream_geometry_t)]
+    g = rdk_stream_geometry_t()
+    _check(L.rdk_stream_geometry(N, n, target_dtype, drafter_dtype, C.byref(g)), "rdk_stream_geometry")
+    return {k: int(getattr(g, k)) for k, _ in rdk_stream_geometry_t._fields_ if k != "reserved"}

@@ -913,9 +913,9 @@ static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
     const int vt = 32 * (int)(16 / es);    // tokens one warp covers with one 16-byte vector per lane
     int C = (N + kSW * 4 * vt - 1) / (kSW * 4 * vt);
     if (C > kMaxGroup) C = kMaxGroup;
-    g.C = C;
     g.nv = (N + C * kSW * vt - 1) / (C * kSW * vt);
     g.Lw = g.nv * vt;
+    g.C = (N + kSW * g.Lw - 1) / (kSW * g.Lw);          // no CTA of a group without tokens
     if ((g.Lw + kSeg - 1) / kSeg > kMaxChunks || (size_t)kSW * g.Lw * es + 16 > 65535) return false;   // slice offsets are 16-bit
     const long long expect = ((long long)n * g.Lw + N - 1) / N;
     long long cap = expect + expect / 8 + 32;
@@ -1045,3 +1045,21 @@ cudaError_t launch_stream_linear(RowParams P, int tz, int ty, int kind, int batc
 }
 
 }  // namespace rdk
+
+extern "C" int rdk_stream_geometry(int32_t N, int32_t n, int32_t target_dtype, int32_t drafter_dtype, rdk_stream_geometry_t* out) {
+    using namespace rdk;
+    if (!out || N < 1 || n < 1 || (target_dtype != RDK_F32 && target_dtype != RDK_BF16) ||
+        (drafter_dtype != RDK_F32 && drafter_dtype != RDK_BF16)) {
+        set_error("rdk_stream_geometry: bad argument");
+        return RDK_ERR_INVALID_ARG;
+    }
+    const size_t es = target_dtype == RDK_F32 ? 4 : 2, ys = drafter_dtype == RDK_F32 ? 4 : 2;
+    StreamGeo g;
+    *out = rdk_stream_geometry_t{};
+    out->supported = N >= kMinStreamN && plan_stream(N, n, es, ys, g) ? 1 : 0;
+    if (!out->supported) return RDK_OK;
+    out->ctas_per_row = g.C; out->warps_per_cta = kSW; out->segment_tokens = g.Lw; out->stages = g.NS;
+    out->live_rows = g.NB; out->cached_slots_per_warp = g.ycap;
+    out->dynamic_shared_bytes = (int64_t)stream_smem(g, es);
+    return RDK_OK;
+}

@@ -100,3 +100,29 @@ def test_binding_refuses_wrong_tensor_types(B):
         B.rdk_prepare_ids(torch.zeros(4, dtype=torch.int64), 16)
     with pytest.raises(TypeError):
         B._dtype_code(torch.zeros(2, dtype=torch.float16))
+
+
+def test_stream_geometry_covers_the_vocabulary_and_fits_shared_memory(B):
+    """Host logic of the streaming kernels' planner: for many shapes the segments cover the vocabulary,
+    there are at most 256 of them, a segment is a whole number of 16-byte vectors per lane, the cache
+    has room for the expected kept tokens of a warp, and the shared memory stays within one SM's."""
+    import paper_2506_03206_b200 as rdk
+    shapes = [(4096, 1), (4096, 4096), (4097, 100), (12808, 2000), (40000, 9000), (128256, 32064), (128256, 12826),
+              (200000, 500), (262144, 32768), (262144, 262144), (400000, 50000)]
+    for N, n in shapes:
+        for tz, ty in ((B.RDK_BF16, B.RDK_BF16), (B.RDK_F32, B.RDK_F32), (B.RDK_BF16, B.RDK_F32)):
+            g = rdk.rdk_stream_geometry(N, n, tz, ty)
+            if not g["supported"]:
+                continue
+            per_vec = 32 * (8 if tz == B.RDK_BF16 else 4)
+            assert g["segment_tokens"] % per_vec == 0
+            segs = g["ctas_per_row"] * g["warps_per_cta"]
+            assert segs * g["segment_tokens"] >= N and segs <= 256 and 1 <= g["ctas_per_row"] <= 16
+            assert (segs - g["warps_per_cta"]) * g["segment_tokens"] < N            # the last CTA is not idle
+            assert 2 <= g["stages"] <= 3 and 3 <= g["live_rows"] <= 5
+            assert g["cached_slots_per_warp"] % 64 == 0 and g["cached_slots_per_warp"] >= 64
+            assert g["dynamic_shared_bytes"] <= 218 * 1024
+    big = rdk.rdk_stream_geometry(128256, 32064)
+    assert big["ctas_per_row"] == 8 and big["segment_tokens"] == 1024      # the benchmark shape
+    assert rdk.rdk_stream_geometry(1000, 10)["supported"] == 0              # small vocabularies take the row kernel
+    assert rdk.rdk_stream_geometry(1 << 21, 1000)["supported"] == 0         # too large for shared memory
