@@ -147,6 +147,11 @@ template <typename TZ> __device__ __forceinline__ float lds_z(uint32_t a);
 template <> __device__ __forceinline__ float lds_z<__nv_bfloat16>(uint32_t a) { return __uint_as_float(lds16(a) << 16); }
 template <> __device__ __forceinline__ float lds_z<float>(uint32_t a) { return __uint_as_float(lds32(a)); }
 
+// one drafter value at shared byte address a, as fp32
+template <typename TY> __device__ __forceinline__ float lds_y1(uint32_t a);
+template <> __device__ __forceinline__ float lds_y1<__nv_bfloat16>(uint32_t a) { return __uint_as_float(lds16(a) << 16); }
+template <> __device__ __forceinline__ float lds_y1<float>(uint32_t a) { return __uint_as_float(lds32(a)); }
+
 // two consecutive drafter values at shared byte address a (aligned to the pair), as fp32
 template <typename TY> __device__ __forceinline__ float2 lds_ypair(uint32_t a);
 template <> __device__ __forceinline__ float2 lds_ypair<__nv_bfloat16>(uint32_t a) {
@@ -392,6 +397,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         const int r0 = __shfl_sync(0xffffffffu, si.r0, 0), kcp = __shfl_sync(0xffffffffu, si.kcp, 0);
         const int kcs = __shfl_sync(0xffffffffu, si.kcs, 0), j0 = __shfl_sync(0xffffffffu, si.j0, 0);
         const int nsteps = (kcs + 63) >> 6;
+        const int si_dummy = __shfl_sync(0xffffffffu, si.dummy, 0);
         const bool ovf = kcp > kcs;
         const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
         const uint32_t yw_off = zslice + 16u + (uint32_t)warp * (uint32_t)g.ystage;
@@ -457,7 +463,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         for (int it = 0; it < rows_g; ++it) {
             const uint32_t zs_a = st_a + zw_off;
             const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(cy) & 15u);      // slot 0 sits this many bytes into the warp's region
-            const uint32_t ys_a = st_a + yw_off + shb + (uint32_t)lane * 2u * (uint32_t)sizeof(TY);   // this lane's pair of step 0
+            const uint32_t ysb_a = st_a + yw_off + shb;                                      // slot 0 of the warp's pair grid
+            const uint32_t ys_a = ysb_a + (uint32_t)lane * 2u * (uint32_t)sizeof(TY);           // this lane's pair of step 0
             mbar_wait(fb, sph, &fail);
 
             // slots that hold no kept token of this segment read as weight 0
@@ -482,20 +489,15 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
 #pragma unroll 4
                 for (int t = lane * kZPer; t < g.Lw; t += 32 * kZPer) mz.push(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)));
             }
+            // Scale of the drafter exponentials: not the maximum of the warp's kept values (finding it first
+            // would hold up every exponential) but one of them, the first; any scale gives the same result
+            // as long as nothing overflows, which the maximum found along the way confirms below.
             float my_w = KIND == RDK_LOGITS ? -INFINITY : 0.f;
-            if (KIND == RDK_LOGITS) {
-#pragma unroll 2
-                for (int st = 0; st < nsteps; ++st) {
-                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)st * 64u * (uint32_t)sizeof(TY));
-                    my_w = fmaxf(my_w, fmaxf(y.x, y.y));
-                }
-                if (ovf)
-                    for (int il = kcs + lane; il < kcp; il += 32) my_w = fmaxf(my_w, to_float<TY>(cy[il]));
-                my_w = warp_max_redux(my_w);
-            }
+            if (KIND == RDK_LOGITS && kcp > si_dummy)
+                my_w = kcs > si_dummy ? lds_y1<TY>(ysb_a + (uint32_t)si_dummy * (uint32_t)sizeof(TY)) : to_float<TY>(cy[si_dummy]);
             const float m_w = warp_max_redux(mz.result());
             const float zoff = m_w > -INFINITY ? -m_w * kLog2e : 0.f;
-            const float yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
+            float yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
 
             // soft-max sweep: sum of e over the segment
             float2 Ea = splat(0.f), Eb = splat(0.f);
@@ -511,8 +513,10 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 }
             }
             // kept tokens: e_z, e_y, their sums; the pairs go to the cache
-            float2 K1 = splat(0.f), Zq = splat(0.f), th = splat(0.f);
-            {
+            float K1s, Zqs, ths, ymax;
+            auto kept_pass = [&]() {
+                float2 K1 = splat(0.f), Zq = splat(0.f), th = splat(0.f);
+                float ym = -INFINITY;
                 const float2 zof = splat(zoff), yof = splat(yoff);
                 const uint32_t cb = cb0 + (uint32_t)par * csz;
 #pragma unroll 2
@@ -522,19 +526,32 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                     const float2 y = lds_ypair<TY>(ys_a + (uint32_t)st * 64u * (uint32_t)sizeof(TY));
                     const float2 ez = ex2_2(ffma2(z, l2e, zof));
                     const float2 ey = KIND == RDK_LOGITS ? ex2_2(ffma2(y, l2e, yof)) : y;
+                    if (KIND == RDK_LOGITS) ym = fmaxf(ym, fmaxf(y.x, y.y));
                     K1 = fadd2(K1, ez); Zq = fadd2(Zq, ey); th = ffma2(ez, ey, th);
                     sts128(cb + (uint32_t)st * 512u, ez.x, ez.y, ey.x, ey.y);
                 }
-            }
-            float E1s = (Ea.x + Ea.y) + (Eb.x + Eb.y), K1s = K1.x + K1.y, Zqs = Zq.x + Zq.y, ths = th.x + th.y;
-            if (ovf) {
-                for (int il = kcs + lane; il < kcp; il += 32) {               // kept tokens beyond the cache
-                    const float ez = ex2(fmaf(lds_z<TZ>(zs_a + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ)), kLog2e, zoff));
-                    const float y = to_float<TY>(cy[il]);
-                    const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
-                    K1s += ez; Zqs += ey; ths = fmaf(ez, ey, ths);
+                K1s = K1.x + K1.y; Zqs = Zq.x + Zq.y; ths = th.x + th.y;
+                if (ovf) {
+                    for (int il = kcs + lane; il < kcp; il += 32) {               // kept tokens beyond the cache
+                        const float ez = ex2(fmaf(lds_z<TZ>(zs_a + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ)), kLog2e, zoff));
+                        const float y = to_float<TY>(cy[il]);
+                        const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
+                        if (KIND == RDK_LOGITS) ym = fmaxf(ym, y);
+                        K1s += ez; Zqs += ey; ths = fmaf(ez, ey, ths);
+                    }
+                }
+                ymax = ym;
+            };
+            kept_pass();
+            if (KIND == RDK_LOGITS) {
+                const float my_true = warp_max_redux(ymax);
+                if (!(my_true - my_w <= 60.f) && my_true > -INFINITY) {     // rare: the reference was a poor scale, take the maximum
+                    my_w = my_true;
+                    yoff = -my_w * kLog2e;
+                    kept_pass();
                 }
             }
+            const float E1s = (Ea.x + Ea.y) + (Eb.x + Eb.y);
             const float tot = warp_sum4(E1s, K1s, Zqs, ths, lane);      // lanes 0, 8, 16, 24 hold the four totals
             // the warp's record goes to the exchange warp, the stage back to the load warp
             if ((lane & 7) == 0) wrec[par][warp][lane >> 3] = tot;
