@@ -187,6 +187,20 @@ def test_many_rows_per_group_every_row_checked():
     _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
 
 
+def test_drafter_values_far_below_their_neighbours():
+    """The streaming kernels scale a warp's drafter exponentials by the first kept value of the warp's
+    range and fall back to the maximum when that value is more than 60 below it: make many such
+    values very small (and some -inf) so that both routes run."""
+    cfg = W.tiny_config(N=30000, n=6000, rows=6, dtype="bf16", trials=4, kept_rule="zipf", zipf_bias=True,
+                        rho=0.8, seed=61)
+    inp = W.make_inputs(cfg)
+    y = inp["drafter"].clone()
+    y[:, ::7] = -250.0
+    y[:, 5::31] = float("-inf")
+    inp["drafter"] = y
+    _run_linear(cfg, inp, check_qtilde=False).assert_ok()
+
+
 def test_few_rows_fewer_than_the_pipeline_depth():
     # one and two rows: the deferred second visits all happen after the row loop
     for rows in (1, 2):
