@@ -188,9 +188,9 @@ def test_many_rows_per_group_every_row_checked():
 
 
 def test_drafter_values_far_below_their_neighbours():
-    """The streaming kernels scale a warp's drafter exponentials by the first kept value of the warp's
-    range and fall back to the maximum when that value is more than 60 below it: make many such
-    values very small (and some -inf) so that both routes run."""
+    """The streaming kernels scale a warp's exponentials by the first value of the warp's range (kept
+    drafter values, target logits) and fall back to the maximum when that value lies far below it: make
+    many such values very small (and some -inf) so that both routes run."""
     cfg = W.tiny_config(N=30000, n=6000, rows=6, dtype="bf16", trials=4, kept_rule="zipf", zipf_bias=True,
                         rho=0.8, seed=61)
     inp = W.make_inputs(cfg)
@@ -198,6 +198,13 @@ def test_drafter_values_far_below_their_neighbours():
     y[:, ::7] = -250.0
     y[:, 5::31] = float("-inf")
     inp["drafter"] = y
+    _run_linear(cfg, inp, check_qtilde=False).assert_ok()
+    # the same for the target logits, whose scale is the first logit of each 1024-token segment
+    z = inp["target"].clone()
+    z[:, ::1024] = -300.0
+    z[:, 2048] = float("-inf")
+    z[:, 5000:5003] = float("-inf")
+    inp["target"] = z
     _run_linear(cfg, inp, check_qtilde=False).assert_ok()
 
 
