@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "4378ea64417149cb325d86fb2757d469bc59b79e9e2525ec21afc3196b6ad9c4",
-               "bytes_per_launch": 102939648 + 3941632}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
+NCU_TRAFFIC = {"sources_sha256": "1e42f9b8b0f8e00e5898eabb6219842d28f7ebf3a3022b92df2c9420b2bfd9ec",
+               "bytes_per_launch": 102952192 + 3322880}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 
