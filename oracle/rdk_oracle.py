@@ -287,14 +287,17 @@ def drafter_qprime(y: np.ndarray, kappa: np.ndarray, N: int, drafter_kind: str) 
 
 def rdk_row(z: np.ndarray, y: np.ndarray, kappa: np.ndarray, u: np.ndarray, mode: str,
             M: np.ndarray | None = None, drafter_kind: str = "logits",
-            operand_bf16: bool = False, w_given: np.ndarray | None = None) -> dict:
+            operand_bf16: bool = False, w_given: np.ndarray | None = None,
+            prior: np.ndarray | None = None) -> dict:
     """Run one row through redistribution, draft draw, rejection test and residual draw.
 
     z [N] target logits, y [n] drafter logits/probabilities, kappa [n] kept ids, u [trials, 4]
     uniforms (lane 0 draft, 1 accept, 2 residual).  mode: "linear" (Eq. rdk-taylor), "exact"
     (M^T q', needs M), or "given" (w_given supplied, e.g. a matrix product computed elsewhere in
     this checker).  operand_bf16 rounds q' at the kept ids to bfloat16 before the exact product
-    (it is then the stored left operand of the contraction).
+    (it is then the stored left operand of the contraction).  prior [N] (linear mode only): logits of
+    the distribution that takes the place of p inside Eq. rdk-taylor (theta and w); verification is
+    against p = softmax(z) all the same.  Without it the formula uses p itself (the literal reading).
     """
     z = np.asarray(z, dtype=F64)
     kappa = np.asarray(kappa, dtype=np.int64)
@@ -307,7 +310,8 @@ def rdk_row(z: np.ndarray, y: np.ndarray, kappa: np.ndarray, u: np.ndarray, mode
     else:
         qp = drafter_qprime(y, kappa, N, drafter_kind)           # O2
         if mode == "linear":
-            theta, w = redistribute_linear(p, qp)                # O3l
+            pi = p if prior is None else softmax(np.asarray(prior, dtype=F64))
+            theta, w = redistribute_linear(pi, qp)               # O3l
         elif mode == "exact":
             valid = (kappa >= 0) & (kappa < N)
             qk = np.where(valid, qp[np.where(valid, kappa, 0)], 0.0)

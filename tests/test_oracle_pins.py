@@ -446,3 +446,33 @@ def test_emit_sequence_bruteforce_and_bonus_distribution():
     u = rng.uniform(size=30000)
     counts = np.bincount([O.emit_sequence([7], [True], [9], p_bonus, x)[-1] for x in u], minlength=6)
     assert np.abs(counts / u.size - p_bonus).max() < 0.012
+
+
+def test_linear_with_a_separate_prior():
+    """Eq. rdk-taylor with a prior pi in place of p.  (i) pi = p is the literal reading, result for
+    result.  (ii) A uniform prior has a closed form that does not involve the target at all:
+    theta = 1/N, q~_j = (N^3 q'_j + 1) / (N^3 + N), S = 1 -- here with a non-uniform target, so the
+    acceptance rate and the residual do see p.  (iii) The output token is still distributed as p."""
+    rng = np.random.default_rng(12)
+    N, n = 12, 5
+    kappa = np.sort(rng.choice(N, n, replace=False))
+    z, y = rng.normal(0, 2, N), rng.normal(0, 2, n)
+    u = rng.random((3, 4))
+    a = O.rdk_row(z, y, kappa, u, "linear")
+    b = O.rdk_row(z, y, kappa, u, "linear", prior=z)
+    for k in ("theta", "S", "alpha", "R"):
+        assert a[k] == b[k]
+    assert np.array_equal(a["w"], b["w"]) and np.array_equal(a["draft"], b["draft"])
+    c = O.rdk_row(z, y, kappa, u, "linear", prior=np.full(N, 0.7))
+    qp = c["qprime"]
+    assert abs(c["theta"] - 1.0 / N) < 1e-15 and abs(c["S"] - 1.0) < 1e-12
+    assert np.allclose(c["qtilde"], (N ** 3 * qp + 1.0) / (N ** 3 + N), rtol=0, atol=1e-15)
+    p = O.softmax(z)
+    assert abs(c["alpha"] - np.minimum(p, c["qtilde"]).sum()) < 1e-15
+    # losslessness: sum_d q~_d a_d = alpha and q~_t a_t + (1 - alpha) r_t = p_t for every token t
+    qt = c["qtilde"]
+    acc = np.minimum(1.0, p / qt)
+    r = np.maximum(0.0, p - qt)
+    r = r / r.sum()
+    assert abs((qt * acc).sum() - c["alpha"]) < 1e-12
+    assert np.allclose(qt * acc + (1 - c["alpha"]) * r, p, rtol=0, atol=1e-12)
