@@ -222,6 +222,25 @@ int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* 
                           void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * rdk_sample_and_verify_prior / rdk_redistribute_linear_prior -- the linear mode with a separate
+ * prior: Eq. "rdk-taylor" uses p both as the direction of the affinity's principal component and
+ * as the distribution to verify against; at draft time the true p is not known yet, so a caller
+ * may supply the logits of a prior pi instead (theta = pi^T q', w_j = (N q'_j + theta pi_j) /
+ * (N + pi_j), pi = softmax(prior)), while the rejection test, alpha and the residual use
+ * p = softmax(target) as always.
+ *   prior             device [rows, N] logits of the same dtype as the target, or one shared row
+ *   prior_row_stride  elements between prior rows; 0 means one row shared by all rows
+ * Everything else as in rdk_sample_and_verify (mode RDK_MODE_LINEAR) and rdk_redistribute_linear.
+ * These calls take the one-CTA-per-row kernel and need no workspace.
+ * ------------------------------------------------------------------------------------------- */
+int rdk_sample_and_verify_prior(const rdk_problem* problem, const void* target, const void* prior,
+                                int64_t prior_row_stride, const void* drafter, const float* uniforms,
+                                int32_t trials, const rdk_outputs* out, void* stream);
+int rdk_redistribute_linear_prior(const rdk_problem* problem, const void* target, const void* prior,
+                                  int64_t prior_row_stride, const void* drafter, float* qtilde_out,
+                                  float* theta_out, float* S_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * rdk_stream_geometry -- host-only query (no CUDA call): how the streaming kernels of the linear
  * mode would lay a problem of N target tokens and n kept ids out, or supported = 0 when such a
  * problem takes the one-CTA-per-row kernel (N < 4096, or shapes beyond shared memory; unsorted

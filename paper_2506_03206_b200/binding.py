@@ -30,7 +30,8 @@ EXPORTS = [
     "rdk_build_affinity_workspace_bytes", "rdk_build_affinity", "rdk_exact_workspace_bytes",
     "rdk_redistribute_exact", "rdk_redistribute_exact_static", "rdk_redistribute_linear",
     "rdk_sample_workspace_bytes", "rdk_sample_and_verify", "rdk_emit_sequences",
-    "rdk_sample_and_verify_host", "rdk_stream_geometry",
+    "rdk_sample_and_verify_host", "rdk_stream_geometry", "rdk_sample_and_verify_prior",
+    "rdk_redistribute_linear_prior",
 ]
 
 
@@ -370,3 +371,59 @@ def rdk_stream_geometry(N: int, n: int, target_dtype: int = RDK_BF16, drafter_dt
     g = rdk_stream_geometry_t()
     _check(L.rdk_stream_geometry(N, n, target_dtype, drafter_dtype, C.byref(g)), "rdk_stream_geometry")
     return {k: int(getattr(g, k)) for k, _ in rdk_stream_geometry_t._fields_ if k != "reserved"}
+
+
+def _prior_stride(prior: torch.Tensor, N: int) -> int:
+    """A [N] prior is one row shared by all rows (stride 0); a [rows, N] prior has its row stride."""
+    if prior.dim() == 1:
+        if prior.numel() != N or not prior.is_contiguous():
+            raise ValueError("a shared prior must be a contiguous [N] tensor")
+        return 0
+    _rows2d(prior, "prior")
+    return prior.stride(0)
+
+
+def rdk_redistribute_linear_prior(index: KeptIndex, target: torch.Tensor, prior: torch.Tensor, drafter: torch.Tensor,
+                                  batch: int, positions: int, drafter_kind: int = RDK_LOGITS):
+    """Eq. rdk-taylor with softmax(prior) in place of p, written out: (q~ [rows, N], theta, S)."""
+    _rows2d(target, "target")
+    _rows2d(drafter, "drafter")
+    if prior.dtype != target.dtype:
+        raise ValueError("the prior must have the target's dtype")
+    rows = batch * positions
+    pb = make_problem(index, target, drafter, batch, positions, drafter_kind)
+    qt = torch.empty(rows, index.N, dtype=torch.float32, device=target.device)
+    theta = torch.empty(rows, dtype=torch.float32, device=target.device)
+    S = torch.empty(rows, dtype=torch.float32, device=target.device)
+    L = lib()
+    L.rdk_redistribute_linear_prior.restype = C.c_int
+    L.rdk_redistribute_linear_prior.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    _check(L.rdk_redistribute_linear_prior(C.byref(pb), target.data_ptr(), prior.data_ptr(), _prior_stride(prior, index.N),
+                                           drafter.data_ptr(), qt.data_ptr(), theta.data_ptr(), S.data_ptr(), _stream()),
+           "rdk_redistribute_linear_prior")
+    return qt, theta, S
+
+
+def rdk_sample_and_verify_prior(index: KeptIndex, target: torch.Tensor, prior: torch.Tensor, drafter: torch.Tensor,
+                                uniforms: torch.Tensor, batch: int, positions: int, drafter_kind: int = RDK_LOGITS,
+                                out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """The linear mode with a separate prior inside Eq. rdk-taylor; verification against softmax(target)."""
+    _rows2d(target, "target")
+    _rows2d(drafter, "drafter")
+    if prior.dtype != target.dtype:
+        raise ValueError("the prior must have the target's dtype")
+    rows = batch * positions
+    trials = uniforms.numel() // (rows * 4)
+    pb = make_problem(index, target, drafter, batch, positions, drafter_kind)
+    if out is None:
+        out = alloc_outputs(rows, batch, trials, target.device)
+    o = outputs_struct(out)
+    L = lib()
+    L.rdk_sample_and_verify_prior.restype = C.c_int
+    L.rdk_sample_and_verify_prior.argtypes = [C.POINTER(rdk_problem), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                              C.c_void_p, C.c_int32, C.POINTER(rdk_outputs), C.c_void_p]
+    _check(L.rdk_sample_and_verify_prior(C.byref(pb), target.data_ptr(), prior.data_ptr(), _prior_stride(prior, index.N),
+                                         drafter.data_ptr(), uniforms.data_ptr(), trials, C.byref(o), _stream()),
+           "rdk_sample_and_verify_prior")
+    return out

@@ -17,6 +17,8 @@ struct RowCtx {
     int N, tid, lane, warp;
     bool zvec, wvec, identity;
     float zoff, inv_zp, yoff, inv_zq, theta, Nf, inv_s;
+    float poff, inv_zpi;      // soft-max of the prior, when there is one
+    bool pvec;
 };
 
 // p and w of the kVec tokens starting at `base` (tokens at or beyond N give p = w = 0).
@@ -51,6 +53,18 @@ __device__ __forceinline__ void load_pw(const RowParams& P, const RowCtx& c, con
         }
     }
 #pragma unroll
+    if (P.prior) {    // Eq. rdk-taylor with the prior's distribution pi in place of p
+        const TZ* prow = static_cast<const TZ*>(P.prior) + (long long)blockIdx.x * P.prior_stride;
+        float pr[kVec];
+        load8<TZ>(prow, base, c.N, c.pvec, -INFINITY, pr);
+#pragma unroll
+        for (int k = 0; k < kVec; ++k) {
+            const float pi = ex2(fmaf(pr[k], kLog2e, c.poff)) * c.inv_zpi;
+            w[k] = (c.Nf * qp[k] + c.theta * pi) / (c.Nf + pi);
+        }
+        return;
+    }
+#pragma unroll
     for (int k = 0; k < kVec; ++k) w[k] = (c.Nf * qp[k] + c.theta * p[k]) / (c.Nf + p[k]);
 }
 
@@ -64,7 +78,7 @@ rdk_row_kernel(const RowParams P) {
     float* seg_w = reinterpret_cast<float*>(cdf_r + num_segs);
     float* seg_r = seg_w + num_segs;
 
-    __shared__ MS red_z[kRowWarps], red_y[kRowWarps], red_t[kRowWarps];
+    __shared__ MS red_z[kRowWarps], red_y[kRowWarps], red_t[kRowWarps], red_p[kRowWarps];
     __shared__ float red_q[kRowWarps];
     __shared__ double red_a[kRowWarps];
     __shared__ float bc[8];
@@ -90,9 +104,13 @@ rdk_row_kernel(const RowParams P) {
     const float* wrow = (MODE == RDK_MODE_PRECOMPUTED_W) ? P.w + (long long)row * P.w_stride : nullptr;
     c.zvec = (reinterpret_cast<uintptr_t>(zrow) & 15u) == 0;
     c.wvec = wrow && (reinterpret_cast<uintptr_t>(wrow) & 15u) == 0;
+    const bool has_prior = MODE == RDK_MODE_LINEAR && P.prior != nullptr;
+    const TZ* prow = has_prior ? static_cast<const TZ*>(P.prior) + (long long)row * P.prior_stride : nullptr;
+    c.pvec = prow && (reinterpret_cast<uintptr_t>(prow) & 15u) == 0;
+    c.poff = 0.f; c.inv_zpi = 1.f;
 
     // ---- pass 1: soft-max statistics (running max / sum), theta numerator ----------------------
-    MS zs{-INFINITY, 0.f, 0.f}, ys{-INFINITY, 0.f, 0.f}, ts{-INFINITY, 0.f, 0.f};
+    MS zs{-INFINITY, 0.f, 0.f}, ys{-INFINITY, 0.f, 0.f}, ts{-INFINITY, 0.f, 0.f}, ps{-INFINITY, 0.f, 0.f};
     float sq = 0.f;
     for (int tile = 0; tile < P.num_tiles; ++tile) {
         const int base = tile * kTile + c.tid * kVec;
@@ -110,14 +128,28 @@ rdk_row_kernel(const RowParams P) {
             float vmax = z[0];
 #pragma unroll
             for (int k = 1; k < kVec; ++k) vmax = fmaxf(vmax, z[k]);
-            if (vmax > -INFINITY) {
+            if (vmax > -INFINITY || MODE == RDK_MODE_LINEAR) {   // (kept drafter values count even where every target logit is -inf)
                 if (vmax > zs.m) {
                     const float sc = ex2((zs.m - vmax) * kLog2e);
                     zs.s *= sc; zs.b *= sc; zs.m = vmax;
                 }
-                const float off = -zs.m * kLog2e;
+                const float off = zs.m > -INFINITY ? -zs.m * kLog2e : 0.f;
 #pragma unroll
                 for (int k = 0; k < kVec; ++k) { e[k] = ex2(fmaf(z[k], kLog2e, off)); zs.s += e[k]; }
+                float pr[kVec], ep[kVec];
+                if (has_prior) {      // the prior's soft-max statistics; theta is then taken with the prior
+                    load8<TZ>(prow, base, P.N, c.pvec, -INFINITY, pr);
+                    float pmax = pr[0];
+#pragma unroll
+                    for (int k = 1; k < kVec; ++k) pmax = fmaxf(pmax, pr[k]);
+                    if (pmax > ps.m) {
+                        const float sc = ex2((ps.m - pmax) * kLog2e);
+                        ps.s *= sc; ps.b *= sc; ps.m = pmax;
+                    }
+                    const float poff = ps.m > -INFINITY ? -ps.m * kLog2e : 0.f;
+#pragma unroll
+                    for (int k = 0; k < kVec; ++k) { ep[k] = ex2(fmaf(pr[k], kLog2e, poff)); ps.s += ep[k]; }
+                }
                 if (MODE == RDK_MODE_LINEAR) {
                     const uint32_t word = __ldg(P.mask + (base >> 5));
                     const int sh = base & 31;
@@ -130,8 +162,8 @@ rdk_row_kernel(const RowParams P) {
                                 const int i = c.identity ? r : __ldg(P.slot + r);
                                 ++r;
                                 const float y = to_float<TY>(yrow[i]);
-                                if (KIND == RDK_LOGITS) { ms_push(ys, y); ms_push(ts, z[k] + y); }
-                                else { sq += y; zs.b += e[k] * y; }
+                                if (KIND == RDK_LOGITS) { ms_push(ys, y); ms_push(ts, (has_prior ? pr[k] : z[k]) + y); }
+                                else { sq += y; if (has_prior) ps.b += ep[k] * y; else zs.b += e[k] * y; }
                             }
                         }
                     }
@@ -144,30 +176,34 @@ rdk_row_kernel(const RowParams P) {
         }
     }
     zs = ms_warp(zs);
+    if (has_prior) ps = ms_warp(ps);
     if (MODE == RDK_MODE_LINEAR) {
         if (KIND == RDK_LOGITS) { ys = ms_warp(ys); ts = ms_warp(ts); }
         else sq = warp_sum(sq);
     }
-    if (c.lane == 0) { red_z[c.warp] = zs; red_y[c.warp] = ys; red_t[c.warp] = ts; red_q[c.warp] = sq; }
+    if (c.lane == 0) { red_z[c.warp] = zs; red_y[c.warp] = ys; red_t[c.warp] = ts; red_q[c.warp] = sq; red_p[c.warp] = ps; }
     __syncthreads();
     if (c.warp == 0) {
         MS a = (c.lane < kRowWarps) ? red_z[c.lane] : MS{-INFINITY, 0.f, 0.f};
         MS b = (c.lane < kRowWarps) ? red_y[c.lane] : MS{-INFINITY, 0.f, 0.f};
         MS t = (c.lane < kRowWarps) ? red_t[c.lane] : MS{-INFINITY, 0.f, 0.f};
         float q = (c.lane < kRowWarps) ? red_q[c.lane] : 0.f;
+        MS pa = (has_prior && c.lane < kRowWarps) ? red_p[c.lane] : MS{-INFINITY, 0.f, 0.f};
         a = ms_warp(a); b = ms_warp(b); t = ms_warp(t); q = warp_sum(q);
+        if (has_prior) pa = ms_warp(pa);
         if (c.lane == 0) {
             float theta = 0.f, zq = 1.f, my = 0.f;
+            const MS pi = has_prior ? pa : a;            // the distribution that enters theta
             if (MODE == RDK_MODE_LINEAR) {
                 if (KIND == RDK_LOGITS) {
                     zq = b.s; my = b.m;
-                    theta = (t.m == -INFINITY) ? 0.f : t.s * ex2((t.m - a.m - b.m) * kLog2e) / (a.s * b.s);
+                    theta = (t.m == -INFINITY) ? 0.f : t.s * ex2((t.m - pi.m - b.m) * kLog2e) / (pi.s * b.s);
                 } else {
                     zq = q;
-                    theta = a.b / (a.s * q);
+                    theta = pi.b / (pi.s * q);
                 }
             }
-            bc[0] = a.m; bc[1] = a.s; bc[2] = my; bc[3] = zq; bc[4] = theta;
+            bc[0] = a.m; bc[1] = a.s; bc[2] = my; bc[3] = zq; bc[4] = theta; bc[6] = pi.m; bc[7] = pi.s;
         }
     }
     __syncthreads();
@@ -176,6 +212,8 @@ rdk_row_kernel(const RowParams P) {
     c.yoff = -bc[2] * kLog2e;
     c.inv_zq = 1.f / bc[3];
     c.theta = bc[4];
+    c.poff = -bc[6] * kLog2e;
+    c.inv_zpi = 1.f / bc[7];
 
     // ---- pass 2: S = sum_j w_j and the per-segment sums of w (done in pass 1 for a given w) -------
     for (int tile = 0; MODE == RDK_MODE_LINEAR && tile < P.num_tiles; ++tile) {
@@ -403,13 +441,14 @@ static bool force_generic_kernel() {
 static int run_rows(const rdk_problem* pb, int mode, const void* target, const void* drafter,
                     const float* w, long long w_stride, const float* uniforms, int trials,
                     const rdk_outputs* out, float* qtilde, float* theta_out, float* S_out,
-                    void* ws, size_t ws_bytes, cudaStream_t s) {
+                    void* ws, size_t ws_bytes, cudaStream_t s, const void* prior = nullptr, long long prior_stride = 0) {
     RowParams P{};
     P.N = pb->N; P.n = pb->n; P.rows = pb->batch * pb->positions; P.trials = trials;
     P.target = target; P.target_stride = pb->target_row_stride ? pb->target_row_stride : pb->N;
     P.drafter = drafter; P.drafter_stride = pb->drafter_row_stride ? pb->drafter_row_stride : pb->n;
     P.w = w; P.w_stride = w_stride ? w_stride : pb->N;
     P.uniforms = uniforms;
+    P.prior = prior; P.prior_stride = prior_stride;
     if (mode == RDK_MODE_LINEAR) {
         KeptIndexView v = make_view(pb->kept_index, pb->N, pb->n);
         P.header = v.header; P.mask = v.mask; P.rank = v.rank; P.slot = v.slot; P.ids = v.ids;
@@ -427,7 +466,7 @@ static int run_rows(const rdk_problem* pb, int mode, const void* target, const v
     cudaError_t e = cudaErrorNotSupported;
     P.positions = pb->positions;
     P.accepted_len = out ? out->accepted_len : nullptr;
-    if (mode == RDK_MODE_LINEAR && trials > 0 && !force_generic_kernel()) {
+    if (mode == RDK_MODE_LINEAR && trials > 0 && !prior && !force_generic_kernel()) {
         e = launch_stream_linear(P, pb->target_dtype, pb->drafter_dtype, pb->drafter_kind, pb->batch, ws, ws_bytes, s);
         if (e == cudaSuccess) return RDK_OK;          // the draw kernel also wrote accepted_len
     }
@@ -459,6 +498,41 @@ extern "C" int rdk_redistribute_linear(const rdk_problem* problem, const void* t
     if (st != RDK_OK) return st;
     return run_rows(problem, RDK_MODE_LINEAR, target, drafter, nullptr, 0, nullptr, 0, nullptr,
                     qtilde_out, theta_out, S_out, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int rdk_redistribute_linear_prior(const rdk_problem* problem, const void* target, const void* prior,
+                                             int64_t prior_row_stride, const void* drafter, float* qtilde_out,
+                                             float* theta_out, float* S_out, void* stream) {
+    int st = validate_problem(problem, "rdk_redistribute_linear_prior", true);
+    if (st != RDK_OK) return st;
+    if (!target || !prior || !drafter || !qtilde_out || (prior_row_stride != 0 && prior_row_stride < problem->N)) {
+        set_error("rdk_redistribute_linear_prior: null pointer or a prior row stride below N");
+        return RDK_ERR_INVALID_ARG;
+    }
+    st = check_arch();
+    if (st != RDK_OK) return st;
+    return run_rows(problem, RDK_MODE_LINEAR, target, drafter, nullptr, 0, nullptr, 0, nullptr,
+                    qtilde_out, theta_out, S_out, nullptr, 0, static_cast<cudaStream_t>(stream), prior, prior_row_stride);
+}
+
+extern "C" int rdk_sample_and_verify_prior(const rdk_problem* problem, const void* target, const void* prior,
+                                           int64_t prior_row_stride, const void* drafter, const float* uniforms,
+                                           int32_t trials, const rdk_outputs* out, void* stream) {
+    int st = validate_problem(problem, "rdk_sample_and_verify_prior", true);
+    if (st != RDK_OK) return st;
+    if (!target || !prior || !drafter || !uniforms || !out || trials < 1 ||
+        (prior_row_stride != 0 && prior_row_stride < problem->N)) {
+        set_error("rdk_sample_and_verify_prior: null pointer, trials < 1 or a prior row stride below N");
+        return RDK_ERR_INVALID_ARG;
+    }
+    if (out->accepted_len && !out->accepted) {
+        set_error("rdk_sample_and_verify_prior: accepted_len needs the accepted output");
+        return RDK_ERR_INVALID_ARG;
+    }
+    st = check_arch();
+    if (st != RDK_OK) return st;
+    return run_rows(problem, RDK_MODE_LINEAR, target, drafter, nullptr, 0, uniforms, trials, out, nullptr,
+                    nullptr, nullptr, nullptr, 0, static_cast<cudaStream_t>(stream), prior, prior_row_stride);
 }
 
 extern "C" size_t rdk_sample_workspace_bytes(const rdk_problem* problem, int32_t mode, int32_t trials) {

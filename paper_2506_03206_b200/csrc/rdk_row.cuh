@@ -13,6 +13,7 @@ struct RowParams {
     const void* drafter; long long drafter_stride;
     const float* w;      long long w_stride;
     const float* uniforms;
+    const void* prior; long long prior_stride;   // logits that replace the target inside Eq. rdk-taylor (NULL: none)
     const int32_t* header; const uint32_t* mask; const int32_t* rank; const int32_t* slot; const int32_t* ids;
     int32_t* draft_token; int32_t* out_token; uint8_t* accepted; float* accept_prob;
     float* alpha; float* theta; float* S; float* residual_mass; float* qtilde;

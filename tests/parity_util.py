@@ -69,7 +69,7 @@ class Tally:
 def compare_sampling(inp: Dict[str, object], out: Dict[str, torch.Tensor], rows: Iterable[int],
                      mode: str, tally: Optional[Tally] = None, M: Optional[np.ndarray] = None,
                      w_given: Optional[np.ndarray] = None, operand_bf16: bool = False,
-                     kept_ids: Optional[np.ndarray] = None) -> Tally:
+                     kept_ids: Optional[np.ndarray] = None, prior=None) -> Tally:
     """Compare rdk_sample_and_verify outputs against the checker for the given rows.
 
     inp: the generator's dict (target, drafter, uniforms, cfg, kept_ids); tensors may live on the GPU.
@@ -86,8 +86,9 @@ def compare_sampling(inp: Dict[str, object], out: Dict[str, torch.Tensor], rows:
         z = to_f64(inp["target"][r])
         y = to_f64(inp["drafter"][r]) if inp.get("drafter") is not None else None
         u = inp["uniforms"][r].cpu().numpy().astype(np.float64)
+        pr = None if prior is None else to_f64(prior if prior.dim() == 1 else prior[r])
         ref = O.rdk_row(z, y, kappa, u, mode, M=M, drafter_kind=cfg.drafter_kind, operand_bf16=operand_bf16,
-                        w_given=None if w_given is None else w_given[idx])
+                        w_given=None if w_given is None else w_given[idx], prior=pr)
         tally.rows += 1
         for name, key in (("alpha", "alpha"), ("S", "S"), ("residual_mass", "R")):
             g = float(o[name][r])

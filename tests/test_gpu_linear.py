@@ -295,3 +295,41 @@ def test_extreme_pruning_heavy_tailed_logits_and_tli_baseline():
     # the first-order formula moves only about theta / N of the mass: both rates agree to ~1e-5 here
     assert torch.all((a_rdk - a_tli).abs() < 1e-4)
     print("T1 mean alpha: RDK(linear)", a_rdk.mean().item(), "TLI", a_tli.mean().item())
+
+
+@pytest.mark.parametrize("dtype,N,n,kind", [("bf16", 5000, 900, "logits"), ("f32", 1001, 77, "logits"),
+                                            ("bf16", 12808, 2000, "probs")])
+def test_linear_with_a_separate_prior(dtype, N, n, kind):
+    """Eq. rdk-taylor with a prior in place of p (per-row priors and one shared prior row), checked
+    against the checker row by row: q~, theta, S element-wise, then draws, rejection test, alpha and
+    residual against the true target."""
+    rdk = _rdk()
+    cfg = W.tiny_config(N=N, n=n, rows=5, dtype=dtype, trials=8, rho=0.7, seed=N + 3, drafter_kind=kind)
+    inp = W.make_inputs(cfg)
+    g = torch.Generator().manual_seed(N)
+    noise = torch.randn(cfg.rows, cfg.N, generator=g) * 1.5
+    per_row = (inp["target"].float() * 0.8 + noise).to(inp["target"].dtype)      # a blurred view of the target
+    shared = per_row[0].clone().contiguous()
+    idx = rdk.rdk_prepare_ids(inp["kept_ids"].cuda(), cfg.N)
+    kappa = inp["kept_ids"].numpy()
+    for prior in (per_row, shared):
+        out = rdk.rdk_sample_and_verify_prior(idx, inp["target"].cuda(), prior.cuda(), inp["drafter"].cuda(),
+                                              inp["uniforms"].cuda(), cfg.batch, cfg.positions, KIND[kind])
+        qt, theta, S = rdk.rdk_redistribute_linear_prior(idx, inp["target"].cuda(), prior.cuda(), inp["drafter"].cuda(),
+                                                         cfg.batch, cfg.positions, KIND[kind])
+        torch.cuda.synchronize()
+        rdk.binding.check_status_word(out)
+        PU.compare_sampling(inp, out, range(cfg.rows), "linear", prior=prior).assert_ok()
+        refs = {}
+        for r in range(cfg.rows):
+            pr = W.to_f64(prior if prior.dim() == 1 else prior[r])
+            refs[r] = O.rdk_row(W.to_f64(inp["target"][r]), W.to_f64(inp["drafter"][r]), kappa, np.zeros((1, 4)), "linear",
+                                drafter_kind=kind, prior=pr)
+            assert PU.close(float(theta[r]), refs[r]["theta"], dtype == "bf16")
+            assert PU.close(float(S[r]), refs[r]["S"], dtype == "bf16")
+        PU.compare_qtilde(qt, refs, dtype == "bf16")
+    # with the target itself as the prior the call reduces to the plain linear mode
+    a = rdk.rdk_sample_and_verify_prior(idx, inp["target"].cuda(), inp["target"].cuda(), inp["drafter"].cuda(),
+                                        inp["uniforms"].cuda(), cfg.batch, cfg.positions, KIND[kind])
+    torch.cuda.synchronize()
+    PU.compare_sampling(inp, a, range(cfg.rows), "linear").assert_ok()
