@@ -268,6 +268,15 @@ def run_ours(args):
             B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, sets[0]["target"], None, w_buf, sets[0]["uniforms"],
                                     cfg.batch, cfg.positions, kind, out=out_list[0], ws=ws)
         launches_per_step = 2 + 2          # operand, contraction; row kernel, accepted length
+    elif args.prior:
+        # Eq. rdk-taylor with one shared prior row (a static stand-in for the unknown target distribution)
+        shared_prior = sets[-1]["target"][0].clone().contiguous()
+
+        def step(i, out_list=outs):
+            s = sets[i % nsets]
+            B.rdk_sample_and_verify_prior(index, s["target"], shared_prior, s["drafter"], s["uniforms"],
+                                          cfg.batch, cfg.positions, kind, out=out_list[i % nsets])
+        launches_per_step = 2              # row kernel, accepted length
     else:
         def step(i, out_list=outs):
             s = sets[i % nsets]
@@ -305,7 +314,7 @@ def run_ours(args):
     B.check_status_word(outs[0], "bench step")
 
     e2e = None
-    if not exact:
+    if not exact and not args.prior:
         # end to end: host (pinned) buffers in, host results out, copies inside the timed region
         e2e_steps = max(3, min(args.steps, 20))
         host_sets = [{k: s[k].cpu().pin_memory() for k in ("target", "drafter", "uniforms")} for s in sets[:2]]
@@ -349,15 +358,19 @@ def run_ours(args):
                                                       NCU_TRAFFIC["sources_sha256"] == _kernel_sources_hash()) else None
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": traffic, "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": algo_bytes,
-                    "peak_source": peak_src, "kernels": "rdk_stream_kernel + rdk_draw_kernel"}
+                    "peak_source": peak_src,
+                    "kernels": "rdk_row_kernel (shared prior)" if args.prior else "rdk_stream_kernel + rdk_draw_kernel"}
+        if args.prior:
+            roofline["traffic"] = None
 
     cpu = None
-    if not args.no_cpu_baseline and not exact:
+    if not args.no_cpu_baseline and not exact and not args.prior:
         cpu_value, cpu_dt, cpu_rows = _cpu_baseline(cfg)
         cpu = {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"{cpu_rows} rows of {args.workload} through oracle.rdk_row (float64 numpy, one thread, {cpu_dt:.1f} s)"}
 
     what = ("exact RDK on tensor cores (bf16 affinity, fp32 accumulate) + sampling/verification" if exact
+            else "linear RDK with one shared prior row in Eq. rdk-taylor + sampling/verification" if args.prior
             else "linear RDK (first-order redistribution + sampling/verification)")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -392,6 +405,9 @@ def main():
                     help="C2 (default) is the benchmark; C3/C4 are the other linear-path sizes, C5 the exact "
                          "tensor-core path (used for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
+    ap.add_argument("--prior", action="store_true",
+                    help="linear workloads: time the variant with a shared static prior inside Eq. rdk-taylor "
+                         "(one-CTA-per-row kernel; no CPU baseline, no end-to-end leg)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
