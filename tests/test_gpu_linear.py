@@ -208,6 +208,14 @@ def test_drafter_values_far_below_their_neighbours():
     _run_linear(cfg, inp, check_qtilde=False).assert_ok()
 
 
+def test_vocabulary_beyond_sixteen_full_groups():
+    # N = 300000: segments of five vectors per lane (the generic sweep), fifteen CTAs per row
+    cfg = W.tiny_config(N=300000, n=2500, rows=3, dtype="bf16", trials=4, kept_rule="zipf", zipf_bias=True,
+                        rho=0.8, seed=71)
+    assert _rdk().rdk_stream_geometry(cfg.N, cfg.n)["segment_tokens"] == 1280
+    _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
+
+
 def test_few_rows_fewer_than_the_pipeline_depth():
     # one and two rows: the deferred second visits all happen after the row loop
     for rows in (1, 2):
