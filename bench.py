@@ -32,7 +32,7 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "1e42f9b8b0f8e00e5898eabb6219842d28f7ebf3a3022b92df2c9420b2bfd9ec",
+NCU_TRAFFIC = {"sources_sha256": "c0ad69b9eccb622de65cbd2af81e630531e694c675c7dbee596a3e092b714459",
                "bytes_per_launch": 102952192 + 3322880}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 

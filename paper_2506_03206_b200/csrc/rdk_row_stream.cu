@@ -299,7 +299,7 @@ template <typename TZ, typename TY, int KIND, int NIT>
 __global__ void __launch_bounds__(kSThreads, 1)
 rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     extern __shared__ __align__(128) unsigned char dsm[];
-    __shared__ __align__(16) float wrec[kMaxNB][kSW][8];   // [row mod NB][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), max z, max y
+    __shared__ __align__(16) float wrec[kMaxNB][kSW][8];   // [row mod NB][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), scale of z, scale of y
     __shared__ __align__(16) float scal[kMaxNB][8];        // [row mod NB]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta
     __shared__ __align__(8) float2 fzy[kMaxNB][kSW];       // [row mod NB][warp]: factors that turn the warp's cached e_z, e_y into p, q'
     __shared__ float akv[kMaxNB][kSW];                     // [row mod NB][warp]: sum of min(p, q~) over the warp's kept tokens
@@ -331,7 +331,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     const float inv_n = 1.f / (float)P.N;
 
     // shared memory: NS stages of [the CTA's slice of a target row | 16 bytes of -inf | one drafter
-    // region per warp], then per warp the (e_z, e_y) cache (two rows) and the gather offsets, then barriers
+    // region per warp], then per warp the (e_z, e_y) cache (NB rows) and the gather offsets, then barriers
     const uint32_t zslice = (uint32_t)kSW * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
     const uint32_t stage = zslice + 16u + (uint32_t)kSW * (uint32_t)g.ystage;
     const uint32_t off_cache = (uint32_t)g.NS * stage;
@@ -365,7 +365,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         }
     }
 
-    // streaming warp w: its own segment; exchange and load warp: lane w looks after warp w's segment
+    // streaming warp w: its own segment; publish, collect and load warp: lane w looks after warp w's segment
     const int seg = crank * kSW + (warp < kSW ? warp : (lane & (kSW - 1)));
     const SegInfo si = seg_info(P, g, seg, n_valid);
     if (warp < kSW) {
@@ -452,7 +452,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             }
         };
 
-        // ---- main loop: first visit of row it, second visit of row it - 1 -------------------------------
+        // ---- main loop: first visit of row it, second visit of row it - (NB - 1) -----------------------
         const TY* cy = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + r0;   // slot 0 of the current row
         int s = 0;
         uint32_t sph = 0, st_a = dsm_a, fb = full_a, eb = empty_a;
@@ -477,7 +477,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 __syncwarp();
             }
 
-            // maxima of the segment and of its kept drafter values
+            // maximum of the segment (the scale of its exponentials)
             uint4 zv[NIT > 0 ? NIT : 1];
             MaxAcc<TZ> mz;
             if (NIT > 0) {
@@ -553,7 +553,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             }
             const float E1s = (Ea.x + Ea.y) + (Eb.x + Eb.y);
             const float tot = warp_sum4(E1s, K1s, Zqs, ths, lane);      // lanes 0, 8, 16, 24 hold the four totals
-            // the warp's record goes to the exchange warp, the stage back to the load warp
+            // the warp's record goes to the publish warp, the stage back to the load warp
             if ((lane & 7) == 0) wrec[par][warp][lane >> 3] = tot;
             if (lane == 0) *reinterpret_cast<float2*>(&wrec[par][warp][4]) = make_float2(m_w, my_w);
             __syncwarp();
