@@ -941,7 +941,7 @@ static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
     cap = (cap + 63) / 64 * 64;
     // The exchange of a row between the CTAs of its group takes about as long as two first visits, so
     // the second visit should trail by several rows: prefer live rows over stages, then give up cache.
-    static const int pref[][2] = {{5, 2}, {4, 2}, {3, 3}, {3, 2}};     // {NB, NS}
+    static const int pref[][2] = {{4, 3}, {5, 2}, {4, 2}, {3, 3}, {3, 2}};     // {NB, NS}, by measured speed
     for (const auto& pr : pref) {
         g.NB = pr[0]; g.NS = pr[1];
         g.ycap = (int)cap;
