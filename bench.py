@@ -32,7 +32,7 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "c0ad69b9eccb622de65cbd2af81e630531e694c675c7dbee596a3e092b714459",
+NCU_TRAFFIC = {"sources_sha256": "2c6e9acaac4c7cedd613525ac4a02bf4651131b0cb5e8f7b3ad2dadc990ab5d3",
                "bytes_per_launch": 102952192 + 3322880}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
