@@ -54,11 +54,11 @@ inline KeptIndexView make_view(const void* base, int N, int n) {
     return v;
 }
 
-// What rdk_prepare_ids learnt about the index it built at `kept_index`: 1 when the kept ids are
-// ascending and all inside [0, N) (rank = drafter index), 0 when not, -1 when this process never
-// built an index at that address.  Kernels that rely on it re-check the header on the device.
-void note_index_order(const void* kept_index, bool ascending_valid);
-int index_order(const void* kept_index);
+// What rdk_prepare_ids learnt about the index it built at `kept_index` for (N, n): 1 when the kept ids
+// are ascending and all inside [0, N) (rank = drafter index), 0 when not, -1 when this process never
+// built an index for that (N, n) at that address.  Kernels that rely on it re-check the header on the device.
+void note_index_order(const void* kept_index, int N, int n, bool ascending_valid);
+int index_order(const void* kept_index, int N, int n);
 
 // ---- host-side error plumbing ------------------------------------------------------------------
 void set_error(const char* fmt, ...);

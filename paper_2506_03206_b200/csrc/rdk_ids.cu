@@ -9,18 +9,20 @@
 namespace rdk {
 
 static std::mutex g_order_mu;
-static std::unordered_map<const void*, bool>& order_map() {
-    static std::unordered_map<const void*, bool> m;
+struct IndexNote { int N, n; bool ascending_valid; };
+static std::unordered_map<const void*, IndexNote>& order_map() {
+    static std::unordered_map<const void*, IndexNote> m;
     return m;
 }
-void note_index_order(const void* kept_index, bool ascending_valid) {
+void note_index_order(const void* kept_index, int N, int n, bool ascending_valid) {
     std::lock_guard<std::mutex> lk(g_order_mu);
-    order_map()[kept_index] = ascending_valid;
+    order_map()[kept_index] = IndexNote{N, n, ascending_valid};
 }
-int index_order(const void* kept_index) {
+int index_order(const void* kept_index, int N, int n) {
     std::lock_guard<std::mutex> lk(g_order_mu);
     auto it = order_map().find(kept_index);
-    return it == order_map().end() ? -1 : (it->second ? 1 : 0);
+    if (it == order_map().end() || it->second.N != N || it->second.n != n) return -1;
+    return it->second.ascending_valid ? 1 : 0;
 }
 
 __global__ void idx_clear_kernel(int32_t* header, uint32_t* mask, int32_t* slot, int words, int N, int n) {
@@ -144,7 +146,7 @@ extern "C" int rdk_prepare_ids(const int32_t* kept_ids, int32_t n, int32_t N, vo
     RDK_CUDA(cudaMemcpyAsync(host_hdr, header, sizeof(host_hdr), cudaMemcpyDeviceToHost, s));
     RDK_CUDA(cudaStreamSynchronize(s));
     if (n_valid_host) *n_valid_host = host_hdr[kHdrValid];
-    note_index_order(kept_index, host_hdr[kHdrIdentity] != 0 && host_hdr[kHdrValid] == n);
+    note_index_order(kept_index, N, n, host_hdr[kHdrIdentity] != 0 && host_hdr[kHdrValid] == n);
     if (host_hdr[kHdrDup]) {
         set_error("rdk_prepare_ids: two drafter indices map to the same target token");
         return RDK_ERR_BAD_IDS;

@@ -280,6 +280,9 @@ struct SegInfo {
     int dummy;          // 1 when slot 0 belongs to the previous segment
     int kcp, kcs;       // slots in use; slots staged and cached
 };
+// The index words are read before anything is known about the header's contents (the host has checked
+// that this index was built for (N, n), so the addresses are good): all look-ups of the set-up then
+// travel together.
 __device__ __forceinline__ SegInfo seg_info(const RowParams& P, const StreamGeo& g, int seg, int n_valid) {
     SegInfo si;
     const long long j0l = (long long)seg * g.Lw;
@@ -314,12 +317,15 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);     // the same in every lane, and the compiler knows it
     const int grp = blockIdx.x / g.C, crank = blockIdx.x % g.C;
 
-    if (!index_matches(P)) {   // same decision in every CTA of the grid; nothing is in flight yet
-        if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
-        return;
-    }
-    const int n_valid = P.header[kHdrValid];
-    if (!P.header[kHdrIdentity] || n_valid != P.n) {   // not the index the host was told about
+    // header and index words of this warp's segment, all requested before any of them is looked at
+    const int4 hdr = __ldg(reinterpret_cast<const int4*>(P.header));            // magic, N, n, valid ids
+    const int hdr_identity = __ldg(P.header + kHdrIdentity);
+    const int n_valid = hdr.w;
+    // streaming warp w: its own segment; publish, collect and load warp: lane w looks after warp w's segment
+    const int seg = crank * kSW + (warp < kSW ? warp : (lane & (kSW - 1)));
+    const SegInfo si = seg_info(P, g, seg, n_valid);
+    if (hdr.x != kIdxMagic || hdr.y != P.N || hdr.z != P.n || !hdr_identity || n_valid != P.n) {
+        // not the index the host was told about: the same decision in every CTA; nothing is in flight yet
         if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
         return;
     }
@@ -365,9 +371,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         }
     }
 
-    // streaming warp w: its own segment; publish, collect and load warp: lane w looks after warp w's segment
-    const int seg = crank * kSW + (warp < kSW ? warp : (lane & (kSW - 1)));
-    const SegInfo si = seg_info(P, g, seg, n_valid);
+    __syncthreads();                        // barriers initialised, padding in place
+
     if (warp < kSW) {
         // ================================ streaming warps ============================================
         const int r0 = si.r0, kcs = si.kcs, j0 = si.j0;
@@ -389,8 +394,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 goff_p[q] = o[0] | (o[1] << 16);
             }
         }
+        __syncwarp();                       // the offsets are the warp's own
     }
-    __syncthreads();
 
     if (warp < kSW) {
         // per-warp quantities, taken from lane 0 so that loops over them are not treated as divergent
@@ -1049,7 +1054,7 @@ cudaError_t launch_stream_linear(RowParams P, int tz, int ty, int kind, int batc
     if ((long long)P.rows * P.trials > 0x7fffffffLL) return cudaErrorNotSupported;
     if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < stream_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
     // ascending, valid kept ids only, as recorded when the index was built (kernel 1 re-checks the header)
-    if (index_order(P.header) != 1) return cudaErrorNotSupported;
+    if (index_order(P.header, P.N, P.n) != 1) return cudaErrorNotSupported;
     StreamGeo g;
     if (!plan_stream(P.N, P.n, es, ys, g)) return cudaErrorNotSupported;
     g.G = 0;
