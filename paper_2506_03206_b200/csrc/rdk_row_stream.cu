@@ -586,6 +586,11 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         // Per row: fold the CTA's 16 warp records into one and publish it in global memory; NB rows
         // later, when the second visits of the row are over, write its per-segment sums.  Lane w < 16
         // looks after warp w; what later steps need of a row is parked in pend[row mod 8].
+        // This grid may have been started while the previous kernel of the stream (the draw kernel of an
+        // earlier call, which may still read the same workspace) was draining.  The streaming and load
+        // warps touch only the inputs and shared memory; this warp and the collect warp do all the
+        // writes to the workspace, so they wait for that kernel here.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         auto finish_row = [&](int itf) {
             const int pf = itf % nb;
             const long long row = grp + (long long)itf * g.G;
@@ -629,6 +634,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         // ================================ collect warp ==================================================
         // Per row: gather the C records of the row from global memory, leave the row scalars and every
         // warp's factors in shared memory for the second visits.
+        asm volatile("griddepcontrol.wait;" ::: "memory");     // see the publish warp
         for (int it = 0; it < rows_g; ++it) {
             const int pc = it % nb;
             const long long row = grp + (long long)it * g.G;
@@ -799,6 +805,7 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
     const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
     const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
     if (!index_matches(P)) return;                 // kernel 1 has reported it
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a following stream kernel may set itself up meanwhile
     asm volatile("griddepcontrol.wait;" ::: "memory");   // kernel 1 (launched just before) is complete and visible
     d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
     d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
@@ -990,12 +997,21 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
     cfg.blockDim = dim3(kSThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;      // the CTAs of a group wait for one another: all must be resident
     attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set itself up while an earlier call's draw kernel drains
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    static thread_local int c_pdl = 1;                // whether the two attributes are accepted together on this system
+    cfg.numAttrs = c_pdl ? 2 : 1;
     e = cudaLaunchKernelEx(&cfg, kern, P, g);
+    if (e != cudaSuccess && c_pdl) {
+        (void)cudaGetLastError();
+        c_pdl = 0;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kern, P, g);
+    }
     if (e != cudaSuccess) return e;
     // small CTAs when the draws of all rows would not be resident at once with large ones (shorter
     // tail), large CTAs otherwise (shorter chain per row)
