@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "2c6e9acaac4c7cedd613525ac4a02bf4651131b0cb5e8f7b3ad2dadc990ab5d3",
-               "bytes_per_launch": 102952192 + 3322880}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
+NCU_TRAFFIC = {"sources_sha256": "5c90040cab2f5f417c5c519fbc1b70ecfff81f66f0f96067a949238c812214e1",
+               "bytes_per_launch": 102943488 + 3922688}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 
