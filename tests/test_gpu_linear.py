@@ -223,6 +223,33 @@ def test_few_rows_fewer_than_the_pipeline_depth():
         _run_linear(cfg, W.make_inputs(cfg), check_qtilde=False).assert_ok()
 
 
+def test_calls_back_to_back_share_one_workspace():
+    """Five calls queued on one stream with no synchronisation between them, all on the same workspace
+    but each with its own inputs and outputs: a call's first kernel may start while the previous call's
+    second kernel is still reading the workspace, and must not disturb it."""
+    rdk = _rdk()
+    B = rdk.binding
+    cfgs = [W.tiny_config(N=36000, n=7000, rows=60, dtype="bf16", trials=2, kept_rule="zipf", zipf_bias=True,
+                          rho=0.8, seed=80 + i) for i in range(5)]
+    inps = [W.make_inputs(c) for c in cfgs]
+    kid = inps[0]["kept_ids"].to("cuda")          # one kept set for all five calls
+    idx = rdk.rdk_prepare_ids(kid, cfgs[0].N)
+    dev = [{k: inp[k].to("cuda") for k in ("target", "drafter", "uniforms")} for inp in inps]
+    ws = None
+    outs = []
+    torch.cuda.synchronize()
+    for c, d in zip(cfgs, dev):
+        o = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, d["target"], d["drafter"], None, d["uniforms"],
+                                      c.batch, c.positions, 0, ws=ws)
+        ws = o["_ws"]
+        outs.append(o)
+    torch.cuda.synchronize()
+    for c, inp, o in zip(cfgs, inps, outs):
+        B.check_status_word(o)
+        PU.compare_sampling(inp, o, range(c.rows), "linear", kept_ids=kid.cpu().numpy()).assert_ok()
+        PU.compare_accepted_len(o, c.batch, c.positions, c.trials)
+
+
 def test_strided_rows_through_the_streaming_kernels():
     """Rows embedded in wider buffers (target stride a multiple of 8 elements, drafter stride even but
     not a multiple of 8, so the drafter rows start at varying 16-byte phases)."""
