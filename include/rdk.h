@@ -209,7 +209,11 @@ int rdk_redistribute_linear(const rdk_problem* problem, const void* target, cons
  *              the linear path, one record of 4160 bytes per row (row scalars and per-segment sums
  *              of w, min(p, q~), max(0, p - q~), p), one counter per (sequence, trial), and 64
  *              bytes per (row, CTA sharing the row) through which those CTAs exchange their
- *              partial soft-max sums.  Its contents need no initialisation.
+ *              partial soft-max sums.  Its contents need no initialisation.  One workspace
+ *              serves one call at a time: calls that share it must be ordered on one stream
+ *              (they may be queued back to back without synchronising).  The call may be
+ *              captured in a CUDA graph and the graph replayed: the second kernel wipes the
+ *              exchanged records, so a replay never meets the previous replay's.
  * Arithmetic of the linear mode: fp32.  For N >= 4096 with ascending kept ids, 16-byte aligned
  * target rows and an even drafter row stride, the quotient 1 / (N + p_j) is expanded in
  * x = p_j / N <= 2^-12 and terms of relative size x^2 (below 2^-24) are dropped; every other

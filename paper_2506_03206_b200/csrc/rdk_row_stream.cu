@@ -901,6 +901,10 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
         }
     }
     __syncthreads();
+    // The records that the CTAs of a group exchanged for this row are spent: wipe them, tags included.
+    // The launches of a replayed graph carry the same tag every time and must not meet their old records.
+    if (t == 0 && tid >= 64 && tid - 64 < (nseg / kSW) * (kXrecBytes / 16))
+        __stcg(reinterpret_cast<uint4*>(P.xrec + (size_t)row * (size_t)(nseg / kSW) * kXrecBytes) + (tid - 64), make_uint4(0u, 0u, 0u, 0u));
     if (tid == 0) {
         const int dtok = res_tok[0];
         const float pd = res_p[0], qd = res_w[0] * d.c.inv_s;
@@ -1053,7 +1057,8 @@ size_t stream_workspace_bytes(int rows, int batch, int trials) {
 }
 
 // A non-zero 32-bit value that differs from the one of every recent call of this process and that
-// stale memory is unlikely to hold.
+// stale memory is unlikely to hold.  (The draw kernel wipes a call's records, so a captured call that
+// is replayed with this same value starts from a workspace without them.)
 static uint32_t next_tag() {
     static std::atomic<uint32_t> ctr{
         (uint32_t)std::chrono::high_resolution_clock::now().time_since_epoch().count() * 0x9E3779B9u + 1u};

@@ -250,6 +250,39 @@ def test_calls_back_to_back_share_one_workspace():
         PU.compare_accepted_len(o, c.batch, c.positions, c.trials)
 
 
+def test_replayed_graph_with_new_inputs_in_the_same_buffers():
+    """One call captured in a CUDA graph and replayed four times, each time with new logits and uniforms
+    copied into the same device buffers: the host's part of the call is frozen in the graph, so whatever
+    tells one launch's records in the workspace from the previous launch's must live on the device."""
+    rdk = _rdk()
+    B = rdk.binding
+    cfgs = [W.tiny_config(N=36000, n=7000, rows=60, dtype="bf16", trials=2, kept_rule="zipf", zipf_bias=True,
+                          rho=0.8, seed=90 + i) for i in range(4)]
+    inps = [W.make_inputs(c) for c in cfgs]
+    c0 = cfgs[0]
+    kid = inps[0]["kept_ids"].to("cuda")          # one kept set for all replays
+    idx = rdk.rdk_prepare_ids(kid, c0.N)
+    buf = {k: inps[0][k].to("cuda").clone() for k in ("target", "drafter", "uniforms")}
+    # a first call outside the capture (one-time set-up of the kernels), then the captured one
+    out = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, buf["target"], buf["drafter"], None, buf["uniforms"],
+                                    c0.batch, c0.positions, 0)
+    ws = out["_ws"]
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, buf["target"], buf["drafter"], None, buf["uniforms"],
+                                  c0.batch, c0.positions, 0, out=out, ws=ws)
+    for c, inp in zip(cfgs, inps):
+        for k in buf:
+            buf[k].copy_(inp[k])
+        graph.replay()
+        torch.cuda.synchronize()
+        B.check_status_word(out)
+        got = {k: v.clone() for k, v in out.items() if v is not None and k != "_ws"}
+        PU.compare_sampling(inp, got, range(c.rows), "linear", kept_ids=kid.cpu().numpy()).assert_ok()
+        PU.compare_accepted_len(got, c.batch, c.positions, c.trials)
+
+
 def test_strided_rows_through_the_streaming_kernels():
     """Rows embedded in wider buffers (target stride a multiple of 8 elements, drafter stride even but
     not a multiple of 8, so the drafter rows start at varying 16-byte phases)."""
