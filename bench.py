@@ -32,7 +32,7 @@ UNIT = "tokens/s"
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "143f30613718644a001aa706a776eeb2aef85ac96bece4f7519a20e32ba41fba",
+NCU_TRAFFIC = {"sources_sha256": "368495009f2b0618217eb5ae984b3a808be9932e751962e2c1759995890eed39",
                "bytes_per_launch": 102941952 + 3496704}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 

@@ -1016,6 +1016,10 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
         cfg.numAttrs = 1;
         e = cudaLaunchKernelEx(&cfg, kern, P, g);
     }
+    if (e == cudaErrorCooperativeLaunchTooLarge) {   // fewer SMs at hand than the device reports: the one-CTA-per-row kernel serves
+        (void)cudaGetLastError();
+        return cudaErrorNotSupported;
+    }
     if (e != cudaSuccess) return e;
     // small CTAs when the draws of all rows would not be resident at once with large ones (shorter
     // tail), large CTAs otherwise (shorter chain per row)
