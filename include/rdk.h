@@ -19,6 +19,11 @@
  *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The library allocates no
  *     device memory and keeps no device state: inputs, outputs, the kept-id index, the affinity
  *     matrix and workspaces are caller-owned and are neither freed nor retained after a call.
+ *     On the HOST the library keeps one small table per process: for every kept-id index that
+ *     rdk_prepare_ids built, its address, (N, n) and whether the ids were ascending and valid.
+ *     rdk_sample_and_verify consults it to pick a kernel; the entries are never removed (a few
+ *     bytes each), and the kernels re-check the index header on the device, so an index buffer
+ *     that was freed and reused for something else is detected, not trusted.
  *   - Calls enqueue work on the caller's cudaStream_t (passed as void*; NULL = default stream) and
  *     return at once; outputs are valid after the stream has been synchronised.  rdk_prepare_ids
  *     and rdk_sample_and_verify_host are the exceptions: they synchronise the stream themselves.
@@ -57,6 +62,14 @@ typedef enum rdk_dtype { RDK_F32 = 0, RDK_BF16 = 1 } rdk_dtype;
 typedef enum rdk_kind { RDK_LOGITS = 0, RDK_PROBS = 1 } rdk_kind;
 typedef enum rdk_mode { RDK_MODE_LINEAR = 0, RDK_MODE_PRECOMPUTED_W = 1 } rdk_mode;
 
+/* rdk_problem.flags.  RDK_FLAG_ROW_KERNEL makes rdk_sample_and_verify take the one-CTA-per-row
+ * kernel even where the streaming kernel would serve (the two can then be compared on the same
+ * inputs; the row kernel divides exactly where the streaming kernel expands 1 / (N + p_j)).      */
+#define RDK_FLAG_ROW_KERNEL 1
+
+/* Which kernel a call of the linear mode takes (see rdk_sample_route).                           */
+typedef enum rdk_route { RDK_ROUTE_ROW_KERNEL = 0, RDK_ROUTE_STREAM_KERNEL = 1 } rdk_route;
+
 /* Physical layouts of the affinity matrix M (n rows i in I, N columns j in T).
  *   RDK_AFF_F32_ROWS : float  M[i * ld + j], ld >= N.           Contracted with fp32 FMAs.
  *   RDK_AFF_BF16_COLS: bf16  Mt[j * ld + i], ld >= n, ld % 8 == 0, base 16-byte aligned
@@ -72,7 +85,7 @@ typedef struct rdk_problem {
     int32_t target_dtype;       /* rdk_dtype of the target logits                                */
     int32_t drafter_dtype;      /* rdk_dtype of the drafter logits / probabilities               */
     int32_t drafter_kind;       /* rdk_kind: RDK_LOGITS are soft-maxed, RDK_PROBS taken as is    */
-    int32_t reserved;           /* must be 0                                                     */
+    int32_t flags;              /* 0, or RDK_FLAG_ROW_KERNEL                                     */
     int64_t target_row_stride;  /* elements between target rows; 0 means N                       */
     int64_t drafter_row_stride; /* elements between drafter rows; 0 means n                      */
     const void* kept_index;     /* device buffer filled by rdk_prepare_ids for this (N, n)       */
@@ -111,8 +124,11 @@ const char* rdk_last_error(void);               /* thread-local detail of the la
  * Sec. 2; ids < 0 or >= N stand for drafter tokens outside the target vocabulary, the set F, and
  * are dropped by the TLI step).  rdk_prepare_ids validates the list and builds, in a caller-owned
  * device buffer of rdk_kept_index_bytes(N, n) bytes (256-byte aligned), a membership bitmask over
- * T with rank counts and the rank -> drafter-index table that the row kernels read.  Any order of
- * ids is accepted; ascending valid ids are the fastest case.
+ * T with rank counts and the rank -> drafter-index table that the row kernels read, and, for
+ * ascending valid ids and N >= 4096, the tables of the streaming kernel (which kept ids fall
+ * into which segment of the vocabulary and where their target logits sit inside a CTA's slice,
+ * for 2-byte and for 4-byte logits; about 4 n bytes + 80 KB).  Any order of ids is accepted;
+ * ascending valid ids are the fastest case.
  *   kept_ids       device int32 [n]
  *   n_valid_host   host int*, may be NULL: receives the number of ids inside [0, N)
  * Synchronises `stream`.  Errors: RDK_ERR_BAD_IDS (duplicate id), RDK_ERR_EMPTY_INTERSECTION,
@@ -205,25 +221,57 @@ int rdk_redistribute_linear(const rdk_problem* problem, const void* target, cons
  *   trials     >= 1 independent draws per row (each uses its own 4 uniforms)
  *   out        see rdk_outputs
  *   ws         device workspace of rdk_sample_workspace_bytes(problem, mode, trials) bytes, 256-byte
- *              aligned (may be NULL when that size is 0).  It holds, between the two kernels of
- *              the linear path, one record of 4160 bytes per row (row scalars and per-segment sums
- *              of w, min(p, q~), max(0, p - q~), p), one counter per (sequence, trial), and 64
- *              bytes per (row, CTA sharing the row) through which those CTAs exchange their
- *              partial soft-max sums.  Its contents need no initialisation.  One workspace
- *              serves one call at a time: calls that share it must be ordered on one stream
- *              (they may be queued back to back without synchronising).  The call may be
- *              captured in a CUDA graph and the graph replayed: the second kernel wipes the
- *              exchanged records, so a replay never meets the previous replay's.
- * Arithmetic of the linear mode: fp32.  For N >= 4096 with ascending kept ids, 16-byte aligned
- * target rows and an even drafter row stride, the quotient 1 / (N + p_j) is expanded in
- * x = p_j / N <= 2^-12 and terms of relative size x^2 (below 2^-24) are dropped; every other
- * problem takes the one-CTA-per-row kernel, which divides.
+ *              aligned (may be NULL when that size is 0).  The streaming kernel keeps there one
+ *              record of 4160 bytes per row (row scalars and per-segment sums of w, min(p, q~),
+ *              max(0, p - q~), p), one 8-byte counter per (sequence, trial), and 64 bytes per
+ *              (row, CTA sharing the row) through which those CTAs exchange their partial
+ *              soft-max sums and tell one another that a row's sums are written.  Its contents
+ *              need no initialisation.  One workspace serves one call at a time: calls that
+ *              share it must be ordered on one stream (they may be queued back to back without
+ *              synchronising).  The call may be captured in a CUDA graph and the graph replayed:
+ *              the kernel wipes the exchanged records of a row once the row is drawn, so a
+ *              replay never meets the previous replay's.
+ * Kernels.  For N >= 4096 with ascending valid kept ids, 16-byte aligned target rows, a 16-byte
+ * aligned drafter base and an even drafter row stride, the linear mode is ONE persistent kernel
+ * (launched cooperatively, one CTA per SM) that streams every row from HBM once; there the
+ * quotient 1 / (N + p_j) is expanded in x = p_j / N <= 2^-12 and terms of relative size x^2
+ * (below 2^-24) are dropped.  Every other problem takes the one-CTA-per-row kernel (three sweeps
+ * over the row, exact division), which is several times slower; rdk_sample_route tells which
+ * one a call would take and why.  The streaming kernel is launched with programmatic stream
+ * serialisation: it may set itself up while the previous kernel of the stream drains, but reads
+ * none of its inputs and touches nothing of the workspace before that kernel is complete, so
+ * inputs written by the kernel queued just before the call are safe.
+ * If a bounded wait inside the kernel expires, out->status_word is set to RDK_ERR_TIMEOUT and the
+ * outputs of that call are not valid.  Arithmetic of the linear mode: fp32.
  * ------------------------------------------------------------------------------------------- */
 size_t rdk_sample_workspace_bytes(const rdk_problem* problem, int32_t mode, int32_t trials);
 int rdk_sample_and_verify(const rdk_problem* problem, int32_t mode, const void* target,
                           const void* drafter, const float* w, int64_t w_row_stride,
                           const float* uniforms, int32_t trials, const rdk_outputs* out,
                           void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * rdk_sample_route -- host-only query (no CUDA call, nothing launched): which kernel
+ * rdk_sample_and_verify would run Algorithm 4 steps 4-8 with for these arguments.  It sees what
+ * rdk_stream_geometry cannot: the flags, alignment and strides of the rows, the workspace, and
+ * whether the kept ids of problem->kept_index were ascending and valid when the index was built.
+ *   why   host const char**, may be NULL: receives a static string naming the first reason the
+ *         streaming kernel cannot serve ("" when it can)
+ * Returns RDK_ROUTE_STREAM_KERNEL or RDK_ROUTE_ROW_KERNEL, or -(rdk_status) for a bad problem.
+ * ------------------------------------------------------------------------------------------- */
+int rdk_sample_route(const rdk_problem* problem, int32_t mode, const void* target,
+                     const void* drafter, int32_t trials, const void* ws, size_t ws_bytes,
+                     const char** why);
+
+/* ---------------------------------------------------------------------------------------------
+ * rdk_test_set_spin_limit -- for tests of the failure path only (the paper has no counterpart).
+ * Every wait inside the streaming kernel (on a shared-memory barrier, on a record another CTA
+ * publishes) gives up after a number of failed tries, records RDK_ERR_TIMEOUT in
+ * out->status_word and lets the kernel run to its end.  This sets that number for later calls of
+ * this process; 0 restores the default (2^20).  With a limit of 1 the waits of an ordinary call
+ * run out, which is how the tests reach the failure path without hanging or faulting anything.
+ * ------------------------------------------------------------------------------------------- */
+void rdk_test_set_spin_limit(uint32_t limit);
 
 /* ---------------------------------------------------------------------------------------------
  * rdk_sample_and_verify_prior / rdk_redistribute_linear_prior -- the linear mode with a separate

@@ -24,6 +24,8 @@ RDK_F32, RDK_BF16 = 0, 1
 RDK_LOGITS, RDK_PROBS = 0, 1
 RDK_MODE_LINEAR, RDK_MODE_PRECOMPUTED_W = 0, 1
 RDK_AFF_F32_ROWS, RDK_AFF_BF16_COLS = 0, 1
+RDK_FLAG_ROW_KERNEL = 1
+RDK_ROUTE_ROW_KERNEL, RDK_ROUTE_STREAM_KERNEL = 0, 1
 
 EXPORTS = [
     "rdk_version", "rdk_status_string", "rdk_last_error", "rdk_kept_index_bytes", "rdk_prepare_ids",
@@ -31,7 +33,7 @@ EXPORTS = [
     "rdk_redistribute_exact", "rdk_redistribute_exact_static", "rdk_redistribute_linear",
     "rdk_sample_workspace_bytes", "rdk_sample_and_verify", "rdk_emit_sequences",
     "rdk_sample_and_verify_host", "rdk_stream_geometry", "rdk_sample_and_verify_prior",
-    "rdk_redistribute_linear_prior",
+    "rdk_redistribute_linear_prior", "rdk_sample_route", "rdk_test_set_spin_limit",
 ]
 
 
@@ -44,7 +46,7 @@ class RdkError(RuntimeError):
 class rdk_problem(C.Structure):
     _fields_ = [("N", C.c_int32), ("n", C.c_int32), ("batch", C.c_int32), ("positions", C.c_int32),
                 ("target_dtype", C.c_int32), ("drafter_dtype", C.c_int32), ("drafter_kind", C.c_int32),
-                ("reserved", C.c_int32), ("target_row_stride", C.c_int64),
+                ("flags", C.c_int32), ("target_row_stride", C.c_int64),
                 ("drafter_row_stride", C.c_int64), ("kept_index", C.c_void_p)]
 
 
@@ -115,6 +117,11 @@ def lib() -> C.CDLL:
                                                  C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                                  C.POINTER(rdk_outputs), C.POINTER(rdk_outputs), C.c_void_p,
                                                  C.c_size_t, C.c_void_p]
+        L.rdk_sample_route.restype = C.c_int
+        L.rdk_sample_route.argtypes = [C.POINTER(rdk_problem), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                       C.c_void_p, C.c_size_t, C.POINTER(C.c_char_p)]
+        L.rdk_test_set_spin_limit.restype = None
+        L.rdk_test_set_spin_limit.argtypes = [C.c_uint32]
         _lib = L
     return _lib
 
@@ -175,13 +182,13 @@ def rdk_prepare_ids(kept_ids: torch.Tensor, N: int) -> KeptIndex:
 
 def make_problem(index: KeptIndex, target: Optional[torch.Tensor], drafter: Optional[torch.Tensor],
                  batch: int, positions: int, drafter_kind: int = RDK_LOGITS,
-                 target_dtype: Optional[int] = None, drafter_dtype: Optional[int] = None) -> rdk_problem:
+                 target_dtype: Optional[int] = None, drafter_dtype: Optional[int] = None, flags: int = 0) -> rdk_problem:
     p = rdk_problem()
     p.N, p.n, p.batch, p.positions = index.N, index.n, batch, positions
     p.target_dtype = _dtype_code(target) if target is not None else (target_dtype or RDK_F32)
     p.drafter_dtype = _dtype_code(drafter) if drafter is not None else (drafter_dtype or RDK_F32)
     p.drafter_kind = drafter_kind
-    p.reserved = 0
+    p.flags = flags
     p.target_row_stride = target.stride(0) if target is not None else 0
     p.drafter_row_stride = drafter.stride(0) if drafter is not None else 0
     p.kept_index = index.buffer.data_ptr()
@@ -304,13 +311,13 @@ def rdk_sample_and_verify(index: KeptIndex, mode: int, target: torch.Tensor,
                           uniforms: torch.Tensor, batch: int, positions: int,
                           drafter_kind: int = RDK_LOGITS,
                           out: Optional[Dict[str, torch.Tensor]] = None,
-                          ws: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+                          ws: Optional[torch.Tensor] = None, flags: int = 0) -> Dict[str, torch.Tensor]:
     _rows2d(target, "target")
     rows = batch * positions
     if uniforms.dtype != torch.float32 or not uniforms.is_contiguous() or uniforms.numel() % (rows * 4):
         raise ValueError("uniforms must be contiguous float32 [rows, trials, 4]")
     trials = uniforms.numel() // (rows * 4)
-    pb = make_problem(index, target, drafter, batch, positions, drafter_kind)
+    pb = make_problem(index, target, drafter, batch, positions, drafter_kind, flags=flags)
     if out is None:
         out = alloc_outputs(rows, batch, trials, target.device)
     o = outputs_struct(out)
@@ -321,6 +328,24 @@ def rdk_sample_and_verify(index: KeptIndex, mode: int, target: torch.Tensor,
                                        C.byref(o), ws.data_ptr(), ws.numel(), _stream()), "rdk_sample_and_verify")
     out["_ws"] = ws        # keep the workspace alive until the stream has consumed it
     return out
+
+
+def rdk_sample_route(index: KeptIndex, mode: int, target: torch.Tensor, drafter: Optional[torch.Tensor],
+                     batch: int, positions: int, trials: int, ws: Optional[torch.Tensor],
+                     drafter_kind: int = RDK_LOGITS, flags: int = 0):
+    """Host-only query: (route, reason) -- which kernel rdk_sample_and_verify would take for these arguments."""
+    pb = make_problem(index, target, drafter, batch, positions, drafter_kind, flags=flags)
+    why = C.c_char_p()
+    r = lib().rdk_sample_route(C.byref(pb), mode, target.data_ptr(), _ptr(drafter), trials, _ptr(ws),
+                               0 if ws is None else ws.numel(), C.byref(why))
+    if r < 0:
+        _check(-r, "rdk_sample_route")
+    return r, (why.value or b"").decode()
+
+
+def rdk_test_set_spin_limit(limit: int) -> None:
+    """Tests of the failure path only: failed tries after which a device-side wait gives up (0 = default)."""
+    lib().rdk_test_set_spin_limit(int(limit))
 
 
 def rdk_emit_sequences(N: int, batch: int, positions: int, bonus_target: torch.Tensor, uniforms: torch.Tensor,

@@ -17,13 +17,41 @@ constexpr int kTile = kRowThreads * kVec;   // tokens one CTA covers per step (4
 constexpr int kSeg = 32 * kVec;             // tokens one warp covers per step (256): one CDF segment
 
 // ---- kept-id index layout (device buffer built by rdk_prepare_ids) ---------------------------
-// [0, 64)            header: int32 magic, N, n, n_valid, dup, identity, ...
-// [64, ..)           uint32 mask[words]    bit t set <=> token t is a kept id inside [0, N)
+// [0, 256)           header: int32 magic, N, n, n_valid, dup, identity, plan, ...
+// [256, ..)          uint32 mask[words]    bit t set <=> token t is a kept id inside [0, N)
 // then               int32  rank[words]    number of set bits in all earlier words
 // then               int32  slot[n]        slot[r] = drafter index of the r-th smallest valid id
 // then               int32  ids[n]         copy of the caller's kept ids
-constexpr int kIdxMagic = 0x52444B31;   // "RDK1"
-enum { kHdrMagic = 0, kHdrN = 1, kHdrn = 2, kHdrValid = 3, kHdrDup = 4, kHdrIdentity = 5 };
+// then, for the target element sizes 2 and 4 bytes (v = 0, 1), the tables of the streaming kernels:
+//                    int4   segdesc[v][256]   per segment: first kept slot r0 (even), kept slots, table start, dummy
+//                    uint16 goff[v][..]       per kept slot: byte offset of its target logit in the CTA's slice
+constexpr int kIdxMagic = 0x52444B32;   // "RDK2"
+enum { kHdrMagic = 0, kHdrN = 1, kHdrn = 2, kHdrValid = 3, kHdrDup = 4, kHdrIdentity = 5, kHdrPlan = 6 };
+
+// ---- segmentation of the vocabulary by the streaming kernels ---------------------------------
+// A row is shared by C CTAs of kStreamWarps warps; warp w of CTA c owns the Lw consecutive tokens
+// ("segment") starting at (c * kStreamWarps + w) * Lw.  Lw is a whole number nv of 16-byte vectors
+// per lane.  Depends on N and the target element size only, so the per-segment tables can be built
+// when the kept ids are prepared.
+#ifndef RDK_STREAM_WARPS
+#define RDK_STREAM_WARPS 16
+#endif
+constexpr int kStreamWarps = RDK_STREAM_WARPS;
+constexpr int kStreamMaxGroup = 16;                              // CTAs that share a row
+constexpr int kStreamMaxSeg = kStreamMaxGroup * kStreamWarps;    // 256
+constexpr int kStreamMinN = 4096;
+struct StreamSegs { int C, Lw, nv; };
+inline bool stream_segments(int N, size_t es, StreamSegs& g) {
+    if (N < kStreamMinN) return false;
+    const int vt = 32 * (int)(16 / es);    // tokens one warp covers with one 16-byte vector per lane
+    int C = (N + 64 * vt - 1) / (64 * vt);     // slices of about 64 vectors per lane (32 KB of logits)
+    if (C > kStreamMaxGroup) C = kStreamMaxGroup;
+    g.nv = (N + C * kStreamWarps * vt - 1) / (C * kStreamWarps * vt);
+    g.Lw = g.nv * vt;
+    g.C = (N + kStreamWarps * g.Lw - 1) / (kStreamWarps * g.Lw);          // no CTA of a group without tokens
+    // offsets into a CTA's slice (and the spare slot behind it) are 16-bit
+    return (size_t)kStreamWarps * g.Lw * es + 16 <= 65535;
+}
 
 struct KeptIndexView {
     const int32_t* header;
@@ -31,6 +59,8 @@ struct KeptIndexView {
     const int32_t* rank;
     const int32_t* slot;
     const int32_t* ids;
+    const int4* segdesc[2];
+    const uint16_t* goff[2];
     int words;
 };
 
@@ -40,7 +70,11 @@ __host__ __device__ inline size_t idx_off_mask() { return 256; }
 __host__ __device__ inline size_t idx_off_rank(int N) { return idx_off_mask() + idx_align(size_t(idx_words(N)) * 4); }
 __host__ __device__ inline size_t idx_off_slot(int N) { return idx_off_rank(N) + idx_align(size_t(idx_words(N)) * 4); }
 __host__ __device__ inline size_t idx_off_ids(int N, int n) { return idx_off_slot(N) + idx_align(size_t(n) * 4); }
-__host__ __device__ inline size_t idx_bytes(int N, int n) { return idx_off_ids(N, n) + idx_align(size_t(n) * 4); }
+// every segment's run of kept slots is padded to a multiple of 64 (and may start one slot early)
+__host__ __device__ inline size_t idx_goff_slots(int n) { return size_t(n) + size_t(kStreamMaxSeg) * 66; }
+__host__ __device__ inline size_t idx_plan_bytes(int n) { return idx_align(size_t(kStreamMaxSeg) * 16) + idx_align(idx_goff_slots(n) * 2); }
+__host__ __device__ inline size_t idx_off_plan(int N, int n, int v) { return idx_off_ids(N, n) + idx_align(size_t(n) * 4) + size_t(v) * idx_plan_bytes(n); }
+__host__ __device__ inline size_t idx_bytes(int N, int n) { return idx_off_plan(N, n, 2); }
 
 inline KeptIndexView make_view(const void* base, int N, int n) {
     const char* b = static_cast<const char*>(base);
@@ -50,6 +84,10 @@ inline KeptIndexView make_view(const void* base, int N, int n) {
     v.rank = reinterpret_cast<const int32_t*>(b + idx_off_rank(N));
     v.slot = reinterpret_cast<const int32_t*>(b + idx_off_slot(N));
     v.ids = reinterpret_cast<const int32_t*>(b + idx_off_ids(N, n));
+    for (int k = 0; k < 2; ++k) {
+        v.segdesc[k] = reinterpret_cast<const int4*>(b + idx_off_plan(N, n, k));
+        v.goff[k] = reinterpret_cast<const uint16_t*>(b + idx_off_plan(N, n, k) + idx_align(size_t(kStreamMaxSeg) * 16));
+    }
     v.words = idx_words(N);
     return v;
 }

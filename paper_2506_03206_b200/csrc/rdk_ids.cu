@@ -99,7 +99,54 @@ __global__ void idx_slot_kernel(const int32_t* __restrict__ ids, const uint32_t*
     if (r != i) atomicExch(&header[kHdrIdentity], 0);
 }
 
-__global__ void idx_seal_kernel(int32_t* header) { header[kHdrMagic] = kIdxMagic; }
+// Tables of the streaming kernels for one target element size (ascending valid ids only: rank =
+// drafter index).  Segment s covers tokens [s Lw, (s + 1) Lw); its kept tokens are the drafter
+// indices [r_lo, r_hi).  The kernels read drafter values in aligned pairs, so the segment's slot
+// grid starts at the even index r0 <= r_lo (slot 0 is a "dummy" of the previous segment when r_lo is
+// odd) and is padded to a multiple of 64 slots.
+// One CTA of kStreamMaxSeg threads: per-segment descriptors {r0, slots in use, table start, dummy}.
+__global__ void idx_segdesc_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ rank,
+                                   int4* segdesc, int N, int n, int Lw) {
+    __shared__ int padded[kStreamMaxSeg];
+    const int s = threadIdx.x;
+    auto rank_at = [&](long long j) -> int {
+        if (j >= N) return n;
+        const uint32_t word = mask[j >> 5];
+        return rank[j >> 5] + __popc(word & ((1u << (j & 31)) - 1u));
+    };
+    const long long j0 = (long long)s * Lw;
+    const int r_lo = rank_at(j0), r_hi = rank_at(j0 + Lw);
+    const int dummy = r_lo & 1, r0 = r_lo - dummy, kcp = r_hi - r0;
+    padded[s] = (kcp + 63) & ~63;
+    __syncthreads();
+    int start = 0;
+    for (int k = 0; k < s; ++k) start += padded[k];
+    segdesc[s] = make_int4(r0, kcp, start, dummy);
+}
+
+// One CTA per segment: byte offset, inside the slice of the CTA that owns the segment, of the
+// target logit of every slot; slots without a kept token of the segment point at the spare
+// element behind the slice, which the kernels keep at weight zero.
+__global__ void idx_goff_kernel(const int32_t* __restrict__ ids, const int4* __restrict__ segdesc,
+                                uint16_t* goff, int N, int Lw, int es) {
+    const int s = blockIdx.x;
+    const int4 d = segdesc[s];
+    const int padded = (d.y + 63) & ~63;
+    const long long j0 = (long long)s * Lw;
+    const int w = s % kStreamWarps;
+    const unsigned spare = (unsigned)kStreamWarps * (unsigned)Lw * (unsigned)es;
+    for (int il = threadIdx.x; il < padded; il += blockDim.x) {
+        unsigned o = spare;
+        if (il < d.y && !(d.w && il == 0))
+            o = ((unsigned)w * (unsigned)Lw + (unsigned)(ids[d.x + il] - j0)) * (unsigned)es;
+        goff[d.z + il] = (uint16_t)o;
+    }
+}
+
+__global__ void idx_seal_kernel(int32_t* header, int plan) {
+    header[kHdrPlan] = plan;
+    header[kHdrMagic] = kIdxMagic;
+}
 
 }  // namespace rdk
 
@@ -155,7 +202,20 @@ extern "C" int rdk_prepare_ids(const int32_t* kept_ids, int32_t n, int32_t N, vo
         set_error("rdk_prepare_ids: no kept id lies inside the target vocabulary [0, %d)", N);
         return RDK_ERR_EMPTY_INTERSECTION;
     }
-    idx_seal_kernel<<<1, 1, 0, s>>>(header);
+    // ascending valid ids: the streaming kernels' tables, for 2-byte and 4-byte target logits
+    int plan = 0;
+    if (host_hdr[kHdrIdentity] != 0 && host_hdr[kHdrValid] == n) {
+        for (int k = 0; k < 2; ++k) {
+            StreamSegs g;
+            const int es = k == 0 ? 2 : 4;
+            if (!stream_segments(N, (size_t)es, g)) continue;
+            int4* sd = const_cast<int4*>(v.segdesc[k]);
+            idx_segdesc_kernel<<<1, kStreamMaxSeg, 0, s>>>(mask, rank, sd, N, n, g.Lw);
+            idx_goff_kernel<<<kStreamMaxSeg, 128, 0, s>>>(ids, sd, const_cast<uint16_t*>(v.goff[k]), N, g.Lw, es);
+            plan |= 1 << k;
+        }
+    }
+    idx_seal_kernel<<<1, 1, 0, s>>>(header, plan);
     RDK_CUDA(cudaGetLastError());
     RDK_CUDA(cudaStreamSynchronize(s));
     return RDK_OK;

@@ -417,8 +417,8 @@ static int validate_problem(const rdk_problem* pb, const char* who, bool need_in
     if ((long long)pb->batch * pb->positions > 0x7fffffffLL) { set_error("%s: too many rows", who); return RDK_ERR_INVALID_ARG; }
     if ((pb->target_dtype != RDK_F32 && pb->target_dtype != RDK_BF16) ||
         (pb->drafter_dtype != RDK_F32 && pb->drafter_dtype != RDK_BF16) ||
-        (pb->drafter_kind != RDK_LOGITS && pb->drafter_kind != RDK_PROBS) || pb->reserved != 0) {
-        set_error("%s: bad dtype / kind / reserved field", who);
+        (pb->drafter_kind != RDK_LOGITS && pb->drafter_kind != RDK_PROBS) || (pb->flags & ~RDK_FLAG_ROW_KERNEL) != 0) {
+        set_error("%s: bad dtype / kind / flags field", who);
         return RDK_ERR_INVALID_ARG;
     }
     if ((pb->target_row_stride != 0 && pb->target_row_stride < pb->N) ||
@@ -429,13 +429,6 @@ static int validate_problem(const rdk_problem* pb, const char* who, bool need_in
     if (need_index && !pb->kept_index) { set_error("%s: kept_index is NULL", who); return RDK_ERR_INVALID_ARG; }
     if (pb->N > kMaxN) { set_error("%s: N=%d exceeds the supported maximum %d", who, pb->N, kMaxN); return RDK_ERR_UNSUPPORTED; }
     return RDK_OK;
-}
-
-// Debugging aid: RDK_FORCE_GENERIC=1 in the environment routes every call to the one-CTA-per-row
-// kernel, so the two kernels can be compared on the same inputs.
-static bool force_generic_kernel() {
-    const char* v = getenv("RDK_FORCE_GENERIC");
-    return v && v[0] == '1';
 }
 
 static int run_rows(const rdk_problem* pb, int mode, const void* target, const void* drafter,
@@ -466,9 +459,9 @@ static int run_rows(const rdk_problem* pb, int mode, const void* target, const v
     cudaError_t e = cudaErrorNotSupported;
     P.positions = pb->positions;
     P.accepted_len = out ? out->accepted_len : nullptr;
-    if (mode == RDK_MODE_LINEAR && trials > 0 && !prior && !force_generic_kernel()) {
+    if (mode == RDK_MODE_LINEAR && trials > 0 && !prior && !(pb->flags & RDK_FLAG_ROW_KERNEL)) {
         e = launch_stream_linear(P, pb->target_dtype, pb->drafter_dtype, pb->drafter_kind, pb->batch, ws, ws_bytes, s);
-        if (e == cudaSuccess) return RDK_OK;          // the draw kernel also wrote accepted_len
+        if (e == cudaSuccess) return RDK_OK;          // the streaming kernel also wrote accepted_len
     }
     if (e == cudaErrorNotSupported)
         e = (mode == RDK_MODE_LINEAR)
@@ -534,6 +527,26 @@ extern "C" int rdk_sample_and_verify_prior(const rdk_problem* problem, const voi
     return run_rows(problem, RDK_MODE_LINEAR, target, drafter, nullptr, 0, uniforms, trials, out, nullptr,
                     nullptr, nullptr, nullptr, 0, static_cast<cudaStream_t>(stream), prior, prior_row_stride);
 }
+
+extern "C" int rdk_sample_route(const rdk_problem* problem, int32_t mode, const void* target, const void* drafter,
+                                int32_t trials, const void* ws, size_t ws_bytes, const char** why) {
+    if (why) *why = "";
+    int st = validate_problem(problem, "rdk_sample_route", mode == RDK_MODE_LINEAR);
+    if (st != RDK_OK) return -st;
+    if (mode != RDK_MODE_LINEAR) { if (why) *why = "precomputed w"; return RDK_ROUTE_ROW_KERNEL; }
+    if (problem->flags & RDK_FLAG_ROW_KERNEL) { if (why) *why = "RDK_FLAG_ROW_KERNEL is set"; return RDK_ROUTE_ROW_KERNEL; }
+    RowParams P{};
+    P.N = problem->N; P.n = problem->n; P.rows = problem->batch * problem->positions; P.trials = trials;
+    P.target = target; P.target_stride = problem->target_row_stride ? problem->target_row_stride : problem->N;
+    P.drafter = drafter; P.drafter_stride = problem->drafter_row_stride ? problem->drafter_row_stride : problem->n;
+    P.header = static_cast<const int32_t*>(problem->kept_index);
+    const char* no = stream_ineligible(P, problem->target_dtype, problem->drafter_dtype, problem->drafter_kind,
+                                       problem->batch, ws, ws_bytes);
+    if (no) { if (why) *why = no; return RDK_ROUTE_ROW_KERNEL; }
+    return RDK_ROUTE_STREAM_KERNEL;
+}
+
+extern "C" void rdk_test_set_spin_limit(uint32_t limit) { set_stream_spin_limit(limit); }
 
 extern "C" size_t rdk_sample_workspace_bytes(const rdk_problem* problem, int32_t mode, int32_t trials) {
     if (!problem || mode != RDK_MODE_LINEAR || trials < 1 || problem->batch < 1 || problem->positions < 1) return 0;

@@ -24,10 +24,9 @@ struct RowParams {
     int32_t* accepted_len;
     float* rec;            // per-row records in the workspace
     int32_t* counters;     // per (sequence, trial) arrival counters in the workspace
-    unsigned char* xrec;   // per (row, CTA of the group) published partial records in the workspace
+    unsigned char* xrec;   // per (row, CTA of the group) published partial records and flags in the workspace
 };
 
-constexpr int kRecFloats = 16 + 4 * 256;  // per-row record: 16 scalars + 4 sums for each of up to 256 segments
 
 // running (max, sum) pair of a soft-max denominator; `b` is a second sum on the same scale
 struct MS { float m, s, b; };
@@ -119,9 +118,13 @@ __device__ __forceinline__ int pick_in_segment(const float (&x)[kVec], float rem
 }
 
 
-// Launches the streaming kernels for the linear path when the problem qualifies; returns
-// cudaErrorNotSupported (and launches nothing) when the generic kernel has to be used.
+// Launches the streaming kernel for the linear path when the problem qualifies; returns
+// cudaErrorNotSupported (and launches nothing) when the one-CTA-per-row kernel has to be used.
 cudaError_t launch_stream_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s);
 size_t stream_workspace_bytes(int rows, int batch, int trials);
+// Why a problem cannot take the streaming kernel (a static string), or NULL when it can.  Host only.
+const char* stream_ineligible(const RowParams& P, int tz, int ty, int kind, int batch, const void* ws, size_t ws_bytes);
+// Failed tries after which a device-side wait of the streaming kernel gives up (0: the default).
+void set_stream_spin_limit(unsigned limit);
 
 }  // namespace rdk

@@ -1,27 +1,32 @@
-// Two-kernel form of the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8) for N >= 4096
-// and kept ids in ascending order.
+// Streaming form of the linear-time path (Eq. rdk-taylor + Algorithm 4 steps 4-8) for N >= 4096
+// and kept ids in ascending order: one persistent kernel, one launch per call.
 //
-// Kernel 1 (rdk_stream_kernel): a persistent grid of G groups of C CTAs, one CTA per SM.  Group g
-// takes rows g, g + G, ...; within a row, streaming warp w of CTA c owns the contiguous token range
-// ("segment") s = 16 c + w.  A CTA has 19 warps and no block-wide barrier in its row loop:
+// The grid is G groups of C CTAs, one CTA per SM.  Group g takes rows g, g + G, ...; within a row,
+// streaming warp w of CTA c owns the contiguous token range ("segment") s = 16 c + w.  A CTA has 20
+// warps and no block-wide barrier in its row loop:
 //   load warp      : per row, one bulk copy (TMA) of the CTA's slice of the target logits and one per
 //                    streaming warp of the matching contiguous run of drafter values, into a ring of
 //                    NS shared-memory stages, so a row is read from HBM exactly once.
-//   16 streaming warps, first visit A(row): maxima, sum of e = exp(z - max) over the segment, and
+//   16 streaming warps, first visit A(row): maximum and sum of e = exp(z - max) over the segment, and
 //                    over the segment's kept tokens sum e_z, sum e_y, sum e_z e_y; the (e_z, e_y)
 //                    pairs are cached.  Second visit B(row), NB - 1 rows later: sum min(p, q~) over
 //                    the cached pairs, when the row's scalars are known.
 //   publish warp   : folds the CTA's 16 warp records of a row into one and publishes it in global
 //                    memory as five 64-bit words, each a value paired with a per-call tag (so every
 //                    word validates itself and no fence is needed); NB rows later, writes the row's
-//                    per-segment sums.
+//                    per-segment sums and raises the CTA's flag for that row.
 //   collect warp   : polls the C records of a row and leaves the row scalars and every warp's scale
 //                    factors in shared memory for the second visits.
+//   draw warp      : CTA c of a group turns rows c, c + C, ... of the group into draws once all C
+//                    flags of the row are up: prefix sums over the segments, locate the segment of the
+//                    draft draw, re-read that one segment (still in L2), pick the token, run the
+//                    rejection test, on rejection the same for the residual draw, write the outputs
+//                    and count the accepted prefix of the sequence.
 // The exchange of a row costs about two first visits of latency; with the second visit trailing by
-// NB - 1 rows and the exchange in warps of its own, it is off the streaming warps' critical path.
-// Kernel 2 (rdk_draw_kernel): one CTA per (row, trial) turns the record into draws: it locates the
-// segment by prefix sums, re-reads that one segment (usually still in L2), picks the token, runs
-// the rejection test and the residual draw, and counts the accepted prefix of each sequence.
+// NB - 1 rows and the exchange and the draws in warps of their own, both are off the streaming
+// warps' critical path.  Everything that depends only on (N, n, kept ids, element size) -- which
+// kept slots belong to which segment and where their target logits sit in the CTA's slice -- is
+// tabulated once by rdk_prepare_ids and read from the kept-id index.
 //
 // Arithmetic, with p = softmax(z), q' = TLI(softmax(y)), x_j = p_j / N <= 2^-12:
 //   w_j = (N q'_j + theta p_j) / (N + p_j) = (q'_j + theta x_j) / (1 + x_j)
@@ -38,18 +43,24 @@
 
 namespace rdk {
 
-constexpr int kSW = 16;                  // warps (= segments) per CTA of kernel 1
-constexpr int kSThreads = (kSW + 3) * 32;   // the streaming warps, the publish warp, the collect warp and the load warp
-constexpr int kMaxGroup = 16;            // CTAs that share a row
-constexpr int kMaxSeg = kMaxGroup * kSW; // 256, matches kRecFloats
-constexpr int kMinStreamN = 4096;
-constexpr unsigned kSpinLimit = 1u << 20;
+constexpr int kSW = kStreamWarps;        // streaming warps (= segments) per CTA
+constexpr int kWPublish = kSW, kWCollect = kSW + 1, kWLoad = kSW + 2;
+constexpr int kSThreads = (kSW + 3) * 32;
+constexpr int kMaxGroup = kStreamMaxGroup;   // CTAs that share a row
+constexpr int kMaxSeg = kStreamMaxSeg;       // 256
+constexpr unsigned kSpinLimitDefault = 1u << 17;   // with up to 2 us per try: a quarter of a second
 constexpr int kMaxChunks = 128;          // 256-token chunks per segment
-constexpr int kMaxNB = 6;                // most rows whose records and caches are alive at once (StreamGeo::NB)
+constexpr int kMaxNB = 8;                // most rows whose records and caches are alive at once (StreamGeo::NB)
+constexpr int kTmemCols = 512;           // tensor memory columns of an SM (128 lanes x 512 columns x 32 bits)
+constexpr int kTmemWarpCols = kTmemCols / (kSW / 4);   // columns of a streaming warp: four warps share a 32-lane quarter
 constexpr int kXrecBytes = 64;           // one published CTA record: five (value, tag) words, padded
+constexpr int kRecFloats = 16 + 4 * kMaxSeg;   // one row's record: 16 scalars, then per segment the sums of w, min(p, q~),
+                                         // max(0, p - q~) and p
+constexpr int kFastNit = 64 / kSW;       // 16-byte vectors per lane in a segment of the common length
+constexpr int kMaxFastSteps = 6;         // kept-token passes of up to this many steps are unrolled, their offsets in registers
 
-// record layout (floats): 16 scalars, then 4 per segment
-enum { kRecOffg = 0, kRecInvZp, kRecYoffg, kRecInvZq, kRecTheta, kRecInvN, kRecInvS, kRecS };
+// scalars of a row's record
+enum { kRecOffg = 0, kRecInvZp, kRecYoffg, kRecInvZq, kRecTheta };
 
 struct Scal { float offg, inv_zp, yoffg, inv_zq, theta, inv_n, inv_s; };
 
@@ -62,7 +73,10 @@ struct StreamGeo {
                            // follows its first visit NB - 1 rows later
     int ycap;              // kept-token slots per warp that are staged and cached (multiple of 64)
     int ystage;            // bytes of a warp's drafter region in a stage
-    uint32_t tag;          // value that marks a record word as written by this call
+    uint32_t tag;          // value that marks a word in the workspace as written by this call
+    unsigned spin_limit;   // failed tries after which a wait gives up
+    const int4* segdesc;   // per segment: first slot r0, slots in use, start in goff[], dummy
+    const uint16_t* goff;  // per slot: byte offset of its target logit in the CTA's slice
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -74,21 +88,10 @@ template <typename T> __device__ __forceinline__ T zero_of();
 template <> __device__ __forceinline__ float zero_of<float>() { return 0.f; }
 template <> __device__ __forceinline__ __nv_bfloat16 zero_of<__nv_bfloat16>() { return __float2bfloat16_rn(0.f); }
 
-// number of kept ids below token j (j may equal N)
-__device__ __forceinline__ int rank_at(const RowParams& P, int j, int n_valid) {
-    if (j >= P.N) return n_valid;
-    const uint32_t word = __ldg(P.mask + (j >> 5));
-    return __ldg(P.rank + (j >> 5)) + __popc(word & ((1u << (j & 31)) - 1u));
-}
-
 // w_j for given p_j and q'_j:  (q' + theta x) (1 - x + x^2),  x = p / N
 __device__ __forceinline__ float taylor_w(const Scal& c, float p, float qp) {
     const float x = p * c.inv_n;
     return fmaf(c.theta, x, qp) * fmaf(x, x - 1.f, 1.f);
-}
-
-__device__ __forceinline__ bool index_matches(const RowParams& P) {
-    return P.header[kHdrMagic] == kIdxMagic && P.header[kHdrN] == P.N && P.header[kHdrn] == P.n;
 }
 
 // ---- packed fp32 pairs ---------------------------------------------------------------------------
@@ -141,16 +144,28 @@ __device__ __forceinline__ uint32_t lds16(uint32_t a) {
 __device__ __forceinline__ void sts128(uint32_t a, float x, float y, float z, float w) {
     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
 }
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+
+// ---- tensor memory as a per-warp scratch-pad -------------------------------------------------------
+// Lane i of a warp reads and writes 32-bit words of TMEM lane 32 (warp % 4) + i; four consecutive columns
+// per access.  Nothing here involves the tensor cores: the 256 KB that would hold MMA accumulators hold
+// the cached (e_z, e_y) pairs of the rows in flight instead, which leaves shared memory to the stages.
+__device__ __forceinline__ void tmem_st4(uint32_t taddr, float a, float b, float c, float d) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(taddr), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)), "r"(__float_as_uint(d)) : "memory");
+}
+__device__ __forceinline__ uint4 tmem_ld4(uint32_t taddr) {
+    uint4 v;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(taddr) : "memory");
+    return v;
+}
 
 // one target logit at shared byte address a, as fp32
 template <typename TZ> __device__ __forceinline__ float lds_z(uint32_t a);
 template <> __device__ __forceinline__ float lds_z<__nv_bfloat16>(uint32_t a) { return __uint_as_float(lds16(a) << 16); }
 template <> __device__ __forceinline__ float lds_z<float>(uint32_t a) { return __uint_as_float(lds32(a)); }
-
-// one drafter value at shared byte address a, as fp32
-template <typename TY> __device__ __forceinline__ float lds_y1(uint32_t a);
-template <> __device__ __forceinline__ float lds_y1<__nv_bfloat16>(uint32_t a) { return __uint_as_float(lds16(a) << 16); }
-template <> __device__ __forceinline__ float lds_y1<float>(uint32_t a) { return __uint_as_float(lds32(a)); }
 
 // two consecutive drafter values at shared byte address a (aligned to the pair), as fp32
 template <typename TY> __device__ __forceinline__ float2 lds_ypair(uint32_t a);
@@ -166,7 +181,6 @@ template <> __device__ __forceinline__ float2 lds_ypair<float>(uint32_t a) {
 // maximum of the 8 logits (bf16) / 4 logits (fp32) in one 16-byte vector
 template <typename TZ> struct MaxAcc;
 template <> struct MaxAcc<float> {
-    static constexpr int kPer = 4;
     float m = -INFINITY;
     __device__ __forceinline__ void push(uint4 q) {
         m = fmaxf(fmaxf(m, __uint_as_float(q.x)), fmaxf(__uint_as_float(q.y), fmaxf(__uint_as_float(q.z), __uint_as_float(q.w))));
@@ -174,24 +188,46 @@ template <> struct MaxAcc<float> {
     __device__ __forceinline__ float result() const { return m; }
 };
 template <> struct MaxAcc<__nv_bfloat16> {
-    static constexpr int kPer = 8;
-    __nv_bfloat162 m2 = __float2bfloat162_rn(-INFINITY);
+    __nv_bfloat162 ma = __float2bfloat162_rn(-INFINITY), mb = __float2bfloat162_rn(-INFINITY);
     __device__ __forceinline__ void push(uint4 q) {
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.y));
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.z));
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+        ma = __hmax2(ma, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
+        mb = __hmax2(mb, *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+        ma = __hmax2(ma, *reinterpret_cast<const __nv_bfloat162*>(&q.z));
+        mb = __hmax2(mb, *reinterpret_cast<const __nv_bfloat162*>(&q.w));
     }
-    __device__ __forceinline__ float result() const { return fmaxf(__low2float(m2), __high2float(m2)); }
+    __device__ __forceinline__ float result() const {
+        const __nv_bfloat162 m2 = __hmax2(ma, mb);
+        return fmaxf(__low2float(m2), __high2float(m2));
+    }
 };
 
-// sum of e = 2^(z log2e + off) over the logits of one 16-byte vector, two packed accumulators
+// 2^t for a pair, t <= 0, on the FMA pipe instead of the special-function unit: t = n + f with n the
+// nearest integer (the low bits of t + 1.5 * 2^23) and |f| <= 1/2, 2^f by a degree-5 polynomial (relative
+// error 2.4e-7, that of ex2.approx), 2^n by adding n to the exponent field.  Below -126 the result is
+// about 1e-38 in place of 0.
+__device__ __forceinline__ float2 ex2_poly2(float2 t) {
+    t.x = fmaxf(t.x, -126.f); t.y = fmaxf(t.y, -126.f);
+    const float2 r = fadd2(t, splat(12582912.f));
+    const float2 n = fadd2(r, splat(-12582912.f));
+    const float2 f = ffma2(n, splat(-1.f), t);
+    float2 p = ffma2(splat(0.001327647129073739f), f, splat(0.009675540961325169f));
+    p = ffma2(p, f, splat(0.05550713092088699f));
+    p = ffma2(p, f, splat(0.24022120237350464f));
+    p = ffma2(p, f, splat(0.6931469440460205f));
+    p = ffma2(p, f, splat(1.0000001192092896f));
+    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23)),
+                       __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23)));
+}
+
+// sum of e = 2^(z log2e + off) over the logits of one 16-byte vector, two packed accumulators.  For bf16
+// logits one pair in four takes the polynomial: the sweep is bound by the special-function unit (16
+// results per clock per SM), and a quarter is what the issue slots have room for.
 template <typename TZ> __device__ __forceinline__ void exp_sum_vec(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb);
 template <> __device__ __forceinline__ void exp_sum_vec<__nv_bfloat16>(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb) {
     const float2 e0 = ex2_2(ffma2(make_float2(bf16_lo(q.x), bf16_hi(q.x)), scale, off));
     const float2 e1 = ex2_2(ffma2(make_float2(bf16_lo(q.y), bf16_hi(q.y)), scale, off));
     const float2 e2 = ex2_2(ffma2(make_float2(bf16_lo(q.z), bf16_hi(q.z)), scale, off));
-    const float2 e3 = ex2_2(ffma2(make_float2(bf16_lo(q.w), bf16_hi(q.w)), scale, off));
+    const float2 e3 = ex2_poly2(ffma2(make_float2(bf16_lo(q.w), bf16_hi(q.w)), scale, off));
     Ea = fadd2(Ea, e0); Eb = fadd2(Eb, e1); Ea = fadd2(Ea, e2); Eb = fadd2(Eb, e3);
 }
 template <> __device__ __forceinline__ void exp_sum_vec<float>(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb) {
@@ -200,23 +236,24 @@ template <> __device__ __forceinline__ void exp_sum_vec<float>(uint4 q, float2 s
     Ea = fadd2(Ea, e0); Eb = fadd2(Eb, e1);
 }
 
-// Wait for the phase of `bar` with the given parity.  BACKOFF > 0: sleep that many nanoseconds after a
-// failed try (the service warps, which are nearly always early, must not eat issue slots while waiting).
-template <int BACKOFF = 0>
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* fail) {
+// Wait for the phase of `bar` with the given parity.  Each try may park the warp in hardware for up to
+// HINT_NS nanoseconds (it wakes as soon as the phase completes), so a waiting warp issues next to nothing;
+// after `limit` failed tries the wait gives up and the host reads RDK_ERR_TIMEOUT.
+template <int HINT_NS = 2000>
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* fail, unsigned limit) {
     unsigned spins = 0;
     uint32_t done = 0;
     while (!done) {
-        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (!done) {
-            if (++spins > kSpinLimit || ((spins & 1023u) == 0 && *reinterpret_cast<volatile int*>(fail))) {
-                atomicExch(fail, 1);      // give up: the host reads RDK_ERR_TIMEOUT
-                break;
-            }
-            if (BACKOFF > 0) __nanosleep(BACKOFF);
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar), "r"(parity), "r"((uint32_t)HINT_NS) : "memory");
+        if (!done && (++spins > limit || *reinterpret_cast<volatile int*>(fail))) {
+            atomicExch(fail, 1);
+            break;
         }
     }
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 // (value, tag) words in global memory: one 64-bit relaxed access each, so a reader sees a value
@@ -236,22 +273,6 @@ __device__ __forceinline__ int ld_volatile_s32(const int* p) {
     return v;
 }
 
-// Combine per-lane partial soft-max records (sum e, sum e_y, sum e e_y on the scales m, my) over
-// the warp; lanes without a record pass m = my = -inf and zeros.
-__device__ __forceinline__ float warp_sum4(float v0, float v1, float v2, float v3, int lane);
-__device__ __forceinline__ float warp_max_redux(float v);
-__device__ __forceinline__ void combine_records(float& E1, float& Zq, float& th, float& m, float& my, int lane) {
-    const float mm = warp_max_redux(m), mmy = warp_max_redux(my);
-    const float f = m > -INFINITY ? ex2((m - mm) * kLog2e) : 0.f;
-    const float g = my > -INFINITY ? ex2((my - mmy) * kLog2e) : 0.f;
-    const float tot = warp_sum4(E1 * f, Zq * g, th * f * g, 0.f, lane);
-    E1 = __shfl_sync(0xffffffffu, tot, 0); Zq = __shfl_sync(0xffffffffu, tot, 8); th = __shfl_sync(0xffffffffu, tot, 16);
-    m = mm; my = mmy;
-}
-
-// ------------------------------------------------------------------------------------------------
-// kernel 1
-// ------------------------------------------------------------------------------------------------
 // Sums of four per-lane values over the warp with 6 shuffles: afterwards lanes 0-7 hold the total of
 // v0, lanes 8-15 of v1, lanes 16-23 of v2, lanes 24-31 of v3.
 __device__ __forceinline__ float warp_sum4(float v0, float v1, float v2, float v3, int lane) {
@@ -273,79 +294,129 @@ __device__ __forceinline__ float warp_max_redux(float v) {
     return m;
 }
 
-// One warp's segment of the vocabulary and the kept tokens inside it.
-struct SegInfo {
-    int j0, len;        // first token, tokens inside [0, N)
-    int r0;             // drafter index of slot 0 of the warp's pair grid (even)
-    int dummy;          // 1 when slot 0 belongs to the previous segment
-    int kcp, kcs;       // slots in use; slots staged and cached
-};
-// The index words are read before anything is known about the header's contents (the host has checked
-// that this index was built for (N, n), so the addresses are good): all look-ups of the set-up then
-// travel together.
-__device__ __forceinline__ SegInfo seg_info(const RowParams& P, const StreamGeo& g, int seg, int n_valid) {
-    SegInfo si;
-    const long long j0l = (long long)seg * g.Lw;
-    si.j0 = (int)(j0l < P.N ? j0l : P.N);
-    si.len = max(0, min(P.N - si.j0, g.Lw));
-    const int r_lo = rank_at(P, si.j0, n_valid), r_hi = rank_at(P, si.j0 + si.len, n_valid);
-    si.dummy = r_lo & 1;
-    si.r0 = r_lo - si.dummy;
-    si.kcp = r_hi - si.r0;
-    si.kcs = min(si.kcp, g.ycap);
-    return si;
+// Combine per-lane partial soft-max records (sum e, sum e_y, sum e e_y on the scales m, my) over
+// the warp; lanes without a record pass m = my = -inf and zeros.
+__device__ __forceinline__ void combine_records(float& E1, float& Zq, float& th, float& m, float& my, int lane) {
+    const float mm = warp_max_redux(m), mmy = warp_max_redux(my);
+    const float f = m > -INFINITY ? ex2((m - mm) * kLog2e) : 0.f;
+    const float g = my > -INFINITY ? ex2((my - mmy) * kLog2e) : 0.f;
+    const float tot = warp_sum4(E1 * f, Zq * g, th * f * g, 0.f, lane);
+    E1 = __shfl_sync(0xffffffffu, tot, 0); Zq = __shfl_sync(0xffffffffu, tot, 8); th = __shfl_sync(0xffffffffu, tot, 16);
+    m = mm; my = mmy;
 }
 
+// ------------------------------------------------------------------------------------------------
+// helpers of the draw kernel (Algorithm 4 steps 4-8)
+// ------------------------------------------------------------------------------------------------
+struct DrawCtx {
+    const void* zrow; const void* yrow; bool zvec;
+    const uint32_t* mask; const int32_t* rank;
+    int N;
+    Scal c;
+};
+
+// p and w of the 8 tokens starting at global token jb (a multiple of 8).  The drafter values of the kept
+// tokens among them are fetched by eight independent loads (tokens that are not kept re-read the first
+// fetched index), so that one round trip serves them all.
+template <typename TZ, typename TY, int KIND>
+__device__ __forceinline__ void draw_pw(const DrawCtx& d, int jb, float (&p)[kVec], float (&w)[kVec]) {
+    float z[kVec];
+    load8<TZ>(static_cast<const TZ*>(d.zrow), jb, d.N, d.zvec, -INFINITY, z);
+    const uint32_t word = __ldg(d.mask + (jb >> 5));
+    const int rbase = __ldg(d.rank + (jb >> 5));          // issued together with the mask and the logits
+    const int sh = jb & 31;
+    const uint32_t mb = (word >> sh) & 0xffu;
+    const int r0 = rbase + __popc(word & ((1u << sh) - 1u));
+    const int rfirst = mb ? r0 : 0;
+    float y[kVec];
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) {
+        const bool kept = (mb >> k) & 1u;
+        const int r = kept ? r0 + __popc(mb & ((1u << k) - 1u)) : rfirst;    // ascending kept ids: rank = drafter index
+        y[k] = to_float<TY>(static_cast<const TY*>(d.yrow)[r]);
+    }
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) {
+        p[k] = ex2(fmaf(z[k], kLog2e, d.c.offg)) * d.c.inv_zp;
+        const bool kept = (mb >> k) & 1u;
+        const float qp = kept ? (KIND == RDK_LOGITS ? ex2(fmaf(y[k], kLog2e, d.c.yoffg)) : y[k]) * d.c.inv_zq : 0.f;
+        w[k] = taylor_w(d.c, p[k], qp);
+    }
+}
+
+enum { kPickW = 0, kPickR = 1, kPickP = 2 };
+
+template <typename TZ, typename TY, int KIND>
+__device__ __forceinline__ void draw_x(const DrawCtx& d, int what, int jb, int seg_end, float (&p)[kVec], float (&w)[kVec], float (&x)[kVec]) {
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) { p[k] = 0.f; w[k] = 0.f; x[k] = 0.f; }
+    if (jb >= seg_end) return;
+    draw_pw<TZ, TY, KIND>(d, jb, p, w);
+#pragma unroll
+    for (int k = 0; k < kVec; ++k)
+        x[k] = what == kPickW ? w[k] : (what == kPickR ? fmaxf(0.f, p[k] - w[k] * d.c.inv_s) : p[k]);
+}
+
+// ------------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------------
 // NIT > 0: a segment is exactly NIT 16-byte vectors per lane, kept in registers between the maximum
 // and the exponential pass; NIT = 0: any segment length, two passes over shared memory.
-template <typename TZ, typename TY, int KIND, int NIT>
+// NST > 0: the kept-token passes take exactly NST steps of 64 slots, unrolled, with the slots' offsets in
+// registers; NST = 0: any number of steps, offsets in shared memory.
+template <typename TZ, typename TY, int KIND, int NIT, int NST>
 __global__ void __launch_bounds__(kSThreads, 1)
 rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     extern __shared__ __align__(128) unsigned char dsm[];
     __shared__ __align__(16) float wrec[kMaxNB][kSW][8];   // [row mod NB][warp]: sum e, sum e_z, sum e_y, sum e_z e_y (kept), scale of z, scale of y
-    __shared__ __align__(16) float scal[kMaxNB][8];        // [row mod NB]: -m log2e, 1/Zp, -my log2e, 1/Zq, theta
+    __shared__ __align__(16) float scal[kMaxNB][8];        // [row mod NB]: theta
     __shared__ __align__(8) float2 fzy[kMaxNB][kSW];       // [row mod NB][warp]: factors that turn the warp's cached e_z, e_y into p, q'
     __shared__ float akv[kMaxNB][kSW];                     // [row mod NB][warp]: sum of min(p, q~) over the warp's kept tokens
     __shared__ __align__(8) unsigned long long abar[kMaxNB];   // [row mod NB]: the 16 warp records of the row are in wrec[]
     __shared__ __align__(8) unsigned long long rbar[kMaxNB];   // [row mod NB]: scal[] and fzy[] of the row are set
     __shared__ __align__(8) unsigned long long bbar[kMaxNB];   // [row mod NB]: akv[] of the row is set
-    __shared__ __align__(8) unsigned long long pbar[8];     // [row mod 8]: the publish warp has parked the row in pend[]
-    __shared__ __align__(16) float pend[8][kSW][8];     // publish and collect warps only, [row mod 8][warp]: the warp's sums, its factors, theta
+    __shared__ __align__(8) unsigned long long pbar[16];    // [row mod 16]: the publish warp has parked the row in pend[]
+    __shared__ __align__(16) float pend[16][kSW][8];    // publish and collect warps only, [row mod 16][warp]: the warp's sums, its factors, theta, a row scalar
     __shared__ int fail;
+    __shared__ uint32_t tmem_base_s;                       // base address of the CTA's tensor memory (unrolled route)
+    constexpr bool kTmem = NST > 0;                        // the pair cache lives in tensor memory, not in shared memory
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);     // the same in every lane, and the compiler knows it
     const int grp = blockIdx.x / g.C, crank = blockIdx.x % g.C;
 
-    // header and index words of this warp's segment, all requested before any of them is looked at
+    // header of the index and this warp's segment descriptor, all requested before any of them is looked at
     const int4 hdr = __ldg(reinterpret_cast<const int4*>(P.header));            // magic, N, n, valid ids
-    const int hdr_identity = __ldg(P.header + kHdrIdentity);
-    const int n_valid = hdr.w;
-    // streaming warp w: its own segment; publish, collect and load warp: lane w looks after warp w's segment
+    const int4 hdr2 = __ldg(reinterpret_cast<const int4*>(P.header) + 1);       // dup, identity, plan
+    // streaming warp w: its own segment; service warps: lane w looks after warp w's segment
     const int seg = crank * kSW + (warp < kSW ? warp : (lane & (kSW - 1)));
-    const SegInfo si = seg_info(P, g, seg, n_valid);
-    if (hdr.x != kIdxMagic || hdr.y != P.N || hdr.z != P.n || !hdr_identity || n_valid != P.n) {
+    const int4 sd = __ldg(g.segdesc + seg);                                     // r0, kcp, start in goff[], dummy
+    if (hdr.x != kIdxMagic || hdr.y != P.N || hdr.z != P.n || !hdr2.y || hdr.w != P.n ||
+        !(hdr2.z & (sizeof(TZ) == 2 ? 1 : 2))) {
         // not the index the host was told about: the same decision in every CTA; nothing is in flight yet
         if (tid == 0 && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_INVALID_ARG);
         return;
     }
-    // the draw kernel may be scheduled already; it waits for this whole grid before reading the records
+    // the next kernel of the stream may be scheduled as soon as this one leaves room; it waits for this
+    // whole grid before it touches its inputs or the workspace
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     constexpr int kZPer = 16 / (int)sizeof(TZ);          // logits per 16 bytes
     const int rows_g = grp < P.rows ? (P.rows - grp + g.G - 1) / g.G : 0;
     const float inv_n = 1.f / (float)P.N;
+    const unsigned spin_limit = g.spin_limit;
 
     // shared memory: NS stages of [the CTA's slice of a target row | 16 bytes of -inf | one drafter
-    // region per warp], then per warp the (e_z, e_y) cache (NB rows) and the gather offsets, then barriers
+    // region per warp], then per warp the (e_z, e_y) cache (NB rows) and (NST = 0) the gather offsets, then barriers
     const uint32_t zslice = (uint32_t)kSW * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
     const uint32_t stage = zslice + 16u + (uint32_t)kSW * (uint32_t)g.ystage;
     const uint32_t off_cache = (uint32_t)g.NS * stage;
     const int nb = g.NB, defer = g.NB - 1;
-    const uint32_t off_goff = off_cache + (uint32_t)kSW * (uint32_t)nb * (uint32_t)g.ycap * 8u;
-    const uint32_t off_bar = off_goff + (uint32_t)kSW * (uint32_t)g.ycap * 2u;
+    const uint32_t off_goff = off_cache + (kTmem ? 0u : (uint32_t)kSW * (uint32_t)nb * (uint32_t)g.ycap * 8u);
+    const uint32_t off_bar = off_goff + (NST > 0 ? 0u : (uint32_t)kSW * (uint32_t)g.ycap * 2u);
     const uint32_t dsm_a = smem_u32(dsm);
     const uint32_t full_a = dsm_a + off_bar, empty_a = full_a + 8u * (uint32_t)g.NS;
+    const int nst = NST > 0 ? NST : g.ycap >> 6;           // steps of 32 lanes x 2 slots in a kept-token pass
 
     if (tid == 0) {
         fail = 0;
@@ -354,86 +425,148 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&rbar[k])));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bbar[k])), "r"(kSW));
         }
-        for (int k = 0; k < 8; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&pbar[k])));
-        for (int k = 0; k < g.NS; ++k) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_a + 8u * k));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_a + 8u * k), "r"(kSW));
-        }
+        for (int k = 0; k < 16; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&pbar[k])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // beyond the vocabulary, and the 16 spare bytes of every stage: weight 0
+    // The load warp sets up the ring's barriers itself and starts the copies of the first rows' target slices
+    // right away (they need nothing from the index), so that HBM's first answer travels while the rest of the
+    // CTA is still setting up.  Only their byte count is announced here; the arrival that completes a stage's
+    // phase follows in the row loop, with the drafter copies.
+    const int pre_rows = min(g.NS, rows_g);
+    if (warp == kWLoad) {
+        if (lane == 0) {
+            for (int k = 0; k < g.NS; ++k) {
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_a + 8u * k));
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_a + 8u * k), "r"(kSW));
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        asm volatile("griddepcontrol.wait;" ::: "memory");     // the inputs may be the previous kernel's outputs
+        if (lane == 0) {
+            const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
+            const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
+            const uint32_t zbytes = (uint32_t)(lenc & ~(kZPer - 1)) * (uint32_t)sizeof(TZ);
+            const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0c;
+            for (int k = 0; k < pre_rows && zbytes; ++k) {
+                const uint32_t fb = full_a + 8u * (uint32_t)k, st_a = dsm_a + (uint32_t)k * stage;
+                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(fb), "r"(zbytes) : "memory");
+                for (uint32_t off = 0; off < zbytes; off += 32768u) {
+                    const uint32_t sz = min(32768u, zbytes - off);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(st_a + off), "l"(reinterpret_cast<const char*>(nz) + off), "r"(sz), "r"(fb) : "memory");
+                }
+                nz += (long long)g.G * P.target_stride;
+            }
+        }
+    }
+    // beyond the vocabulary, and the 16 spare bytes of every stage: weight 0; the drafter regions start
+    // out as weight 0 too (slots beyond a copy keep whatever an earlier row left there, and are masked)
     {
         const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
         const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
+        const TY yfill = KIND == RDK_LOGITS ? neg_inf<TY>() : zero_of<TY>();
+        const int ycount = kSW * g.ystage / (int)sizeof(TY);
         for (int k = 0; k < g.NS; ++k) {
             TZ* zs = reinterpret_cast<TZ*>(dsm + (size_t)k * stage);
             for (int t = lenc + tid; t < kSW * g.Lw + kZPer; t += kSThreads) zs[t] = neg_inf<TZ>();
+            TY* ysr = reinterpret_cast<TY*>(dsm + (size_t)k * stage + zslice + 16u);
+            for (int t = tid; t < ycount; t += kSThreads) ysr[t] = yfill;
         }
     }
 
-    __syncthreads();                        // barriers initialised, padding in place
+    // per-warp quantities of the streaming warps (taken from lane 0 so that the compiler knows they are uniform)
+    const int w_r0 = __shfl_sync(0xffffffffu, sd.x, 0), w_kcp = __shfl_sync(0xffffffffu, sd.y, 0);
+    const int w_gstart = __shfl_sync(0xffffffffu, sd.z, 0), w_dummy = __shfl_sync(0xffffffffu, sd.w, 0);
+    const int w_kcs = min(w_kcp, g.ycap);
+    const uint32_t pad2 = zslice | (zslice << 16);      // both slots at the spare -inf
+
+    // offsets (from the start of the slice, 16 bits each) of the target logits of this lane's two slots of every step
+    uint32_t gor[NST > 0 ? NST : 1];
+    if (warp < kSW) {
+        const uint32_t* gt = reinterpret_cast<const uint32_t*>(g.goff + w_gstart);
+        const int npairs = ((w_kcp + 63) & ~63) >> 1;       // pairs tabulated for this segment
+        if (NST > 0) {
+#pragma unroll
+            for (int st = 0; st < (NST > 0 ? NST : 1); ++st) {
+                const int q = st * 32 + lane;
+                uint32_t o = q < npairs ? __ldg(gt + q) : pad2;
+                if (2 * q >= w_kcs) o = (o & 0xffff0000u) | zslice;            // beyond the cache: uncached route
+                if (2 * q + 1 >= w_kcs) o = (o & 0x0000ffffu) | (zslice << 16);
+                gor[st] = o;
+            }
+        } else {
+            const uint32_t gbase = dsm_a + off_goff + (uint32_t)warp * (uint32_t)g.ycap * 2u;
+            for (int q = lane; q < nst * 32; q += 32) {
+                uint32_t o = q < npairs ? __ldg(gt + q) : pad2;
+                if (2 * q >= w_kcs) o = (o & 0xffff0000u) | zslice;
+                if (2 * q + 1 >= w_kcs) o = (o & 0x0000ffffu) | (zslice << 16);
+                sts32(gbase + (uint32_t)q * 4u, o);
+            }
+            gor[0] = 0u;
+        }
+    }
+
+    if (kTmem && warp == 0) {
+        // all 512 columns: one CTA per SM (a kernel that asks for tensor memory on the same SM waits until this
+        // one has given it back)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();                        // barriers initialised, padding and tables in place, tensor memory allocated
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
     if (warp < kSW) {
         // ================================ streaming warps ============================================
-        const int r0 = si.r0, kcs = si.kcs, j0 = si.j0;
-        const int nsteps = (kcs + 63) >> 6;                 // steps of 32 lanes x 2 slots
-        const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);   // the warp's segment within the slice
-        // shared byte offset (from the start of the slice, 16 bits) of the target logit of every cached
-        // slot; slots that hold no kept token of this segment point at the spare -inf
-        {
-            uint32_t* goff_p = reinterpret_cast<uint32_t*>(dsm + off_goff + (size_t)warp * g.ycap * 2);
-            for (int q = lane; q < nsteps * 32; q += 32) {
-                uint32_t o[2];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int il = 2 * q + h;
-                    o[h] = zslice;
-                    if (il < kcs && !(si.dummy && il == 0))
-                        o[h] = zw_off + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ);
-                }
-                goff_p[q] = o[0] | (o[1] << 16);
-            }
-        }
-        __syncwarp();                       // the offsets are the warp's own
-    }
-
-    if (warp < kSW) {
-        // per-warp quantities, taken from lane 0 so that loops over them are not treated as divergent
-        const int r0 = __shfl_sync(0xffffffffu, si.r0, 0), kcp = __shfl_sync(0xffffffffu, si.kcp, 0);
-        const int kcs = __shfl_sync(0xffffffffu, si.kcs, 0), j0 = __shfl_sync(0xffffffffu, si.j0, 0);
-        const int nsteps = (kcs + 63) >> 6;
-        const int si_dummy = __shfl_sync(0xffffffffu, si.dummy, 0);
+        const int r0 = w_r0, kcp = w_kcp, kcs = w_kcs;
+        const int j0 = (int)min((long long)seg * g.Lw, (long long)P.N);
         const bool ovf = kcp > kcs;
         const uint32_t zw_off = (uint32_t)warp * (uint32_t)g.Lw * (uint32_t)sizeof(TZ);
         const uint32_t yw_off = zslice + 16u + (uint32_t)warp * (uint32_t)g.ystage;
         const uint32_t csz = (uint32_t)g.ycap * 8u;
         const uint32_t cb0 = dsm_a + off_cache + (uint32_t)warp * (uint32_t)nb * csz + (uint32_t)lane * 16u;
+        // tensor memory: this warp's quarter of the lanes (warp % 4), its 128 columns there, 4 columns per step and live row
+        const uint32_t tb0 = tmem_base_s + ((uint32_t)(warp & 3) << 21) + (uint32_t)(warp >> 2) * (uint32_t)kTmemWarpCols;
+        constexpr int kRowCols = 4 * (NST > 0 ? NST : 1);
         const uint32_t gl = dsm_a + off_goff + (uint32_t)warp * (uint32_t)g.ycap * 2u + (uint32_t)lane * 4u;
-        // this lane's slots of the pair grid that hold no kept token of the segment (slot 0 when it belongs
-        // to the previous segment, and the tail of the last step), as element indices, -1 = none
-        const int pad_a = (si.dummy && lane == 0 && kcs > 0) ? 0 : -1;
-        const int pad_b = kcs + lane < nsteps * 64 ? kcs + lane : -1;
-        const int pad_c = kcs + lane + 32 < nsteps * 64 ? kcs + lane + 32 : -1;
+        // slot il = 64 st + 2 lane + h of the pair grid holds a kept token of the segment iff il < kcs, and
+        // il > 0 or slot 0 is not the previous segment's; lim > 64 st + h says the first
+        const int lim = kcs - 2 * lane;
+        const bool last_step = NST > 1 && kcs > (NST - 1) * 64;      // the last of the NST steps holds slots of this warp
+        const bool skip0 = w_dummy && lane == 0;
         const long long ystep = (long long)g.G * P.drafter_stride;
         const float2 l2e = splat(kLog2e);
 
-        // ---- second visit of local row `itb`: sum of min(p, q~) over the cached kept tokens -----------
-        auto second_visit = [&](int itb, int par, uint32_t ph) {       // par = itb mod NB, ph = parity of itb / NB
-            mbar_wait(smem_u32(&rbar[par]), ph, &fail);
+        // ---- second visit of a row: sum of min(p, q~) over the cached kept tokens ----------------------
+        // sv_sum: this lane's share, once the row's scalars are in place (par = row mod NB)
+        auto sv_sum = [&](int itb, int par) -> float {
             const float theta = scal[par][4];
             const float2 f = fzy[par][warp];                  // p = f.x e_z,  q' = f.y e_y
             // q~ = q' + x (theta - q'),  x = p / N
             const float2 fz2 = splat(f.x), fy2 = splat(f.y), xs2 = splat(f.x * inv_n), th2 = splat(theta), neg1 = splat(-1.f);
             float2 ak2 = splat(0.f);
             const uint32_t cb = cb0 + (uint32_t)par * csz;
-#pragma unroll 2
-            for (int st = 0; st < nsteps; ++st) {
-                const uint4 c4 = lds128(cb + (uint32_t)st * 512u);
+            auto sv_math = [&](uint4 c4) {
                 const float2 ez = make_float2(__uint_as_float(c4.x), __uint_as_float(c4.y));
                 const float2 ey = make_float2(__uint_as_float(c4.z), __uint_as_float(c4.w));
                 const float2 p = fmul2(ez, fz2), qp = fmul2(ey, fy2), x = fmul2(ez, xs2);
                 const float2 w = ffma2(x, ffma2(qp, neg1, th2), qp);
                 ak2 = fadd2(ak2, make_float2(fminf(p.x, w.x), fminf(p.y, w.y)));
+            };
+            if (NST > 0) {
+                // all loads first (tensor memory answers asynchronously), then the arithmetic
+                uint4 c4[NST > 0 ? NST : 1];
+#pragma unroll
+                for (int st = 0; st < (NST > 0 ? NST : 1); ++st)
+                    if (st < NST - 1 || NST == 1 || last_step) c4[st] = tmem_ld4(tb0 + (uint32_t)(par * kRowCols + st * 4));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int st = 0; st < (NST > 0 ? NST : 1); ++st)
+                    if (st < NST - 1 || NST == 1 || last_step) sv_math(c4[st]);
+            } else {
+#pragma unroll 2
+                for (int st = 0; st < nst; ++st) sv_math(lds128(cb + (uint32_t)st * 512u));
             }
             float ak = ak2.x + ak2.y;
             if (ovf) {   // kept tokens beyond the cache: from global memory again
@@ -450,10 +583,13 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                     ak += fminf(p, fmaf(p * inv_n, theta - qp, qp));
                 }
             }
+            return ak;
+        };
+        auto sv_finish = [&](int par, float ak) {
             ak = warp_sum(ak);
             if (lane == 0) {
                 akv[par][warp] = ak;
-                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bbar[par])) : "memory");
+                mbar_arrive(smem_u32(&bbar[par]));
             }
         };
 
@@ -461,45 +597,33 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         const TY* cy = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + r0;   // slot 0 of the current row
         int s = 0;
         uint32_t sph = 0, st_a = dsm_a, fb = full_a, eb = empty_a;
-        unsigned char* st_p = dsm;
         int par = 0;                                     // it mod NB
         int bit = 0, bpar = 0;                           // next row to get its second visit, the same mod NB
         uint32_t bph = 0;
-        for (int it = 0; it < rows_g; ++it) {
+        auto first_visit = [&]() {
             const uint32_t zs_a = st_a + zw_off;
             const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(cy) & 15u);      // slot 0 sits this many bytes into the warp's region
             const uint32_t ysb_a = st_a + yw_off + shb;                                      // slot 0 of the warp's pair grid
             const uint32_t ys_a = ysb_a + (uint32_t)lane * 2u * (uint32_t)sizeof(TY);           // this lane's pair of step 0
-            mbar_wait(fb, sph, &fail);
-
-            // slots that hold no kept token of this segment read as weight 0
-            {
-                TY* yp = reinterpret_cast<TY*>(st_p + yw_off + shb);
-                const TY fill = KIND == RDK_LOGITS ? neg_inf<TY>() : zero_of<TY>();
-                if (pad_a >= 0) yp[pad_a] = fill;
-                if (pad_b >= 0) yp[pad_b] = fill;
-                if (pad_c >= 0) yp[pad_c] = fill;
-                __syncwarp();
-            }
 
             // maximum of the segment (the scale of its exponentials)
             uint4 zv[NIT > 0 ? NIT : 1];
             MaxAcc<TZ> mz;
             if (NIT > 0) {
 #pragma unroll
-                for (int k = 0; k < NIT; ++k) zv[k] = lds128(zs_a + (uint32_t)(k * 32 + lane) * 16u);
+                for (int k = 0; k < (NIT > 0 ? NIT : 1); ++k) zv[k] = lds128(zs_a + (uint32_t)(k * 32 + lane) * 16u);
 #pragma unroll
-                for (int k = 0; k < NIT; ++k) mz.push(zv[k]);
+                for (int k = 0; k < (NIT > 0 ? NIT : 1); ++k) mz.push(zv[k]);
             } else {
 #pragma unroll 4
                 for (int t = lane * kZPer; t < g.Lw; t += 32 * kZPer) mz.push(lds128(zs_a + (uint32_t)t * (uint32_t)sizeof(TZ)));
             }
             // Scale of the drafter exponentials: not the maximum of the warp's kept values (finding it first
             // would hold up every exponential) but one of them, the first; any scale gives the same result
-            // as long as nothing overflows, which the maximum found along the way confirms below.
+            // as long as nothing grows too large, which the sum found along the way confirms below.
             float my_w = KIND == RDK_LOGITS ? -INFINITY : 0.f;
-            if (KIND == RDK_LOGITS && kcp > si_dummy)
-                my_w = kcs > si_dummy ? lds_y1<TY>(ysb_a + (uint32_t)si_dummy * (uint32_t)sizeof(TY)) : to_float<TY>(cy[si_dummy]);
+            if (KIND == RDK_LOGITS && kcp > w_dummy)
+                my_w = kcs > w_dummy ? lds_z<TY>(ysb_a + (uint32_t)w_dummy * (uint32_t)sizeof(TY)) : to_float<TY>(cy[w_dummy]);
             const float m_w = warp_max_redux(mz.result());
             const float zoff = m_w > -INFINITY ? -m_w * kLog2e : 0.f;
             float yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
@@ -510,7 +634,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 const float2 of = splat(zoff);
                 if (NIT > 0) {
 #pragma unroll
-                    for (int k = 0; k < NIT; ++k) exp_sum_vec<TZ>(zv[k], l2e, of, Ea, Eb);
+                    for (int k = 0; k < (NIT > 0 ? NIT : 1); ++k) exp_sum_vec<TZ>(zv[k], l2e, of, Ea, Eb);
                 } else {
 #pragma unroll 4
                     for (int t = lane * kZPer; t < g.Lw; t += 32 * kZPer)
@@ -518,41 +642,61 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 }
             }
             // kept tokens: e_z, e_y, their sums; the pairs go to the cache
-            float K1s, Zqs, ths, ymax;
+            float K1s, Zqs, ths;
+            const uint32_t cbA = cb0 + (uint32_t)par * csz;
+            auto kept_step = [&](int st, uint32_t go, float2 zof, float2 yof, float2& K1, float2& Zq, float2& th) {
+                const float2 z = make_float2(lds_z<TZ>(st_a + (go & 0xffffu)), lds_z<TZ>(st_a + (go >> 16)));
+                const float2 y = lds_ypair<TY>(ys_a + (uint32_t)st * 64u * (uint32_t)sizeof(TY));
+                const bool v0 = (lim > st * 64) && !(st == 0 && skip0), v1 = lim > st * 64 + 1;
+                const float2 ez = ex2_2(ffma2(z, l2e, zof));
+                float2 ey;
+                if (KIND == RDK_LOGITS) {
+                    float2 t = ffma2(y, l2e, yof);
+                    t.x = v0 ? t.x : -INFINITY; t.y = v1 ? t.y : -INFINITY;
+                    ey = ex2_2(t);
+                } else {
+                    ey = make_float2(v0 ? y.x : 0.f, v1 ? y.y : 0.f);
+                }
+                K1 = fadd2(K1, ez); Zq = fadd2(Zq, ey); th = ffma2(ez, ey, th);
+                if (kTmem) tmem_st4(tb0 + (uint32_t)(par * kRowCols + st * 4), ez.x, ez.y, ey.x, ey.y);
+                else sts128(cbA + (uint32_t)st * 512u, ez.x, ez.y, ey.x, ey.y);
+            };
             auto kept_pass = [&]() {
                 float2 K1 = splat(0.f), Zq = splat(0.f), th = splat(0.f);
-                float ym = -INFINITY;
                 const float2 zof = splat(zoff), yof = splat(yoff);
-                const uint32_t cb = cb0 + (uint32_t)par * csz;
+                if (NST > 0) {
+#pragma unroll
+                    for (int st = 0; st < (NST > 0 ? NST : 1); ++st)
+                        if (st < NST - 1 || NST == 1 || last_step) kept_step(st, gor[st], zof, yof, K1, Zq, th);
+                } else {
 #pragma unroll 2
-                for (int st = 0; st < nsteps; ++st) {
-                    const uint32_t go = lds32(gl + (uint32_t)st * 128u);
-                    const float2 z = make_float2(lds_z<TZ>(st_a + (go & 0xffffu)), lds_z<TZ>(st_a + (go >> 16)));
-                    const float2 y = lds_ypair<TY>(ys_a + (uint32_t)st * 64u * (uint32_t)sizeof(TY));
-                    const float2 ez = ex2_2(ffma2(z, l2e, zof));
-                    const float2 ey = KIND == RDK_LOGITS ? ex2_2(ffma2(y, l2e, yof)) : y;
-                    if (KIND == RDK_LOGITS) ym = fmaxf(ym, fmaxf(y.x, y.y));
-                    K1 = fadd2(K1, ez); Zq = fadd2(Zq, ey); th = ffma2(ez, ey, th);
-                    sts128(cb + (uint32_t)st * 512u, ez.x, ez.y, ey.x, ey.y);
+                    for (int st = 0; st < nst; ++st) kept_step(st, lds32(gl + (uint32_t)st * 128u), zof, yof, K1, Zq, th);
                 }
                 K1s = K1.x + K1.y; Zqs = Zq.x + Zq.y; ths = th.x + th.y;
+                if (kTmem) asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 if (ovf) {
                     for (int il = kcs + lane; il < kcp; il += 32) {               // kept tokens beyond the cache
                         const float ez = ex2(fmaf(lds_z<TZ>(zs_a + (uint32_t)(__ldg(P.ids + r0 + il) - j0) * (uint32_t)sizeof(TZ)), kLog2e, zoff));
                         const float y = to_float<TY>(cy[il]);
                         const float ey = KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, yoff)) : y;
-                        if (KIND == RDK_LOGITS) ym = fmaxf(ym, y);
                         K1s += ez; Zqs += ey; ths = fmaf(ez, ey, ths);
                     }
                 }
-                ymax = ym;
             };
             kept_pass();
             if (KIND == RDK_LOGITS) {
-                const float my_true = warp_max_redux(ymax);
-                if (!(my_true - my_w <= 60.f) && my_true > -INFINITY) {     // rare: the reference was a poor scale, take the maximum
-                    my_w = my_true;
-                    yoff = -my_w * kLog2e;
+                // 2^64 and beyond (or not a number), or the first value was -inf: a poor scale, take the maximum
+                const bool poor = kcp > w_dummy && !(my_w > -INFINITY);
+                if (poor || __any_sync(0xffffffffu, !(Zqs < 1.8e19f))) {
+                    float ym = -INFINITY;
+                    for (int st = 0; st < nst; ++st) {
+                        const float2 y = lds_ypair<TY>(ys_a + (uint32_t)st * 64u * (uint32_t)sizeof(TY));
+                        const bool v0 = (lim > st * 64) && !(st == 0 && skip0), v1 = lim > st * 64 + 1;
+                        ym = fmaxf(ym, fmaxf(v0 ? y.x : -INFINITY, v1 ? y.y : -INFINITY));
+                    }
+                    if (ovf) for (int il = kcs + lane; il < kcp; il += 32) ym = fmaxf(ym, to_float<TY>(cy[il]));
+                    my_w = warp_max_redux(ym);
+                    yoff = my_w > -INFINITY ? -my_w * kLog2e : 0.f;
                     kept_pass();
                 }
             }
@@ -563,41 +707,46 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             if (lane == 0) *reinterpret_cast<float2*>(&wrec[par][warp][4]) = make_float2(m_w, my_w);
             __syncwarp();
             if (lane == 0) {
-                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&abar[par])) : "memory");
-                asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(eb) : "memory");
+                mbar_arrive(smem_u32(&abar[par]));
+                mbar_arrive(eb);
             }
-
+        };
+        for (int it = 0; it < rows_g; ++it) {
+            mbar_wait(fb, sph, &fail, spin_limit);
+            first_visit();
             if (it >= defer) {
-                second_visit(bit, bpar, bph);
+                mbar_wait(smem_u32(&rbar[bpar]), bph, &fail, spin_limit);
+                sv_finish(bpar, sv_sum(bit, bpar));
                 ++bit;
                 if (++bpar == nb) { bpar = 0; bph ^= 1u; }
             }
             if (++par == nb) par = 0;
             cy += ystep;
-            st_a += stage; st_p += stage; fb += 8u; eb += 8u;
-            if (++s == g.NS) { s = 0; sph ^= 1u; st_a = dsm_a; st_p = dsm; fb = full_a; eb = empty_a; }
+            st_a += stage; fb += 8u; eb += 8u;
+            if (++s == g.NS) { s = 0; sph ^= 1u; st_a = dsm_a; fb = full_a; eb = empty_a; }
         }
         for (; bit < rows_g; ++bit) {
-            second_visit(bit, bpar, bph);
+            mbar_wait(smem_u32(&rbar[bpar]), bph, &fail, spin_limit);
+            sv_finish(bpar, sv_sum(bit, bpar));
             if (++bpar == nb) { bpar = 0; bph ^= 1u; }
         }
-    } else if (warp == kSW) {
+    } else if (warp == kWPublish) {
         // ================================ publish warp ==================================================
         // Per row: fold the CTA's 16 warp records into one and publish it in global memory; NB rows
-        // later, when the second visits of the row are over, write its per-segment sums.  Lane w < 16
-        // looks after warp w; what later steps need of a row is parked in pend[row mod 8].
-        // This grid may have been started while the previous kernel of the stream (the draw kernel of an
-        // earlier call, which may still read the same workspace) was draining.  The streaming and load
-        // warps touch only the inputs and shared memory; this warp and the collect warp do all the
-        // writes to the workspace, so they wait for that kernel here.
+        // later, when the second visits of the row are over, write its per-segment sums for the draw
+        // kernel.  Lane w < 16 looks after warp w; what later steps need of a row is parked in
+        // pend[row mod 16].
+        // This grid may have been started while the previous kernel of the stream was draining: nothing
+        // of the workspace and none of the inputs is touched before that kernel is complete.
         asm volatile("griddepcontrol.wait;" ::: "memory");
         auto finish_row = [&](int itf) {
             const int pf = itf % nb;
             const long long row = grp + (long long)itf * g.G;
-            mbar_wait<100>(smem_u32(&bbar[pf]), (uint32_t)((itf / nb) & 1), &fail);
+            mbar_wait(smem_u32(&bbar[pf]), (uint32_t)((itf / nb) & 1), &fail, spin_limit);
+            float* rec = P.rec + row * kRecFloats;
             if (lane < kSW) {
-                const float4 w0 = *reinterpret_cast<const float4*>(&pend[itf & 7][lane][0]);
-                const float4 f4 = *reinterpret_cast<const float4*>(&pend[itf & 7][lane][4]);     // fz, fy, theta (from the collect warp)
+                const float4 w0 = *reinterpret_cast<const float4*>(&pend[itf & 15][lane][0]);
+                const float4 f4 = *reinterpret_cast<const float4*>(&pend[itf & 15][lane][4]);     // fz, fy, theta, a row scalar (from the collect warp)
                 const float theta = f4.z, ak = akv[pf][lane];
                 // sums over the segment: p; w of the not-kept tokens (theta x); w of the kept tokens from the moments
                 const float segP = w0.x * f4.x;
@@ -605,32 +754,34 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 const float oov = theta * xs * fmaxf(0.f, w0.x - w0.y);
                 const float Kw = f4.y * w0.z - f4.y * xs * w0.w + theta * xs * w0.y;
                 const float a_s = oov + ak;
-                reinterpret_cast<float4*>(P.rec + row * kRecFloats + 16)[seg] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP - a_s), segP);
+                reinterpret_cast<float4*>(rec + 16)[seg] = make_float4(oov + Kw, a_s, fmaxf(0.f, segP - a_s), segP);
+                if (crank == 0 && lane < 5) rec[lane] = lane == 4 ? theta : f4.w;     // -m log2e, 1/Zp, -my log2e, 1/Zq, theta
             }
         };
         for (int it = 0; it < rows_g + nb; ++it) {
             if (it < rows_g) {
                 const int par = it % nb;
                 const long long row = grp + (long long)it * g.G;
-                mbar_wait<100>(smem_u32(&abar[par]), (uint32_t)((it / nb) & 1), &fail);
+                mbar_wait(smem_u32(&abar[par]), (uint32_t)((it / nb) & 1), &fail, spin_limit);
                 float E1 = 0.f, Zq = 0.f, th = 0.f, m = -INFINITY, my = -INFINITY, K1 = 0.f;
                 if (lane < kSW) {
                     const volatile float* wr = &wrec[par][lane][0];
                     E1 = wr[0]; K1 = wr[1]; Zq = wr[2]; th = wr[3]; m = wr[4]; my = wr[5];
-                    *reinterpret_cast<float4*>(&pend[it & 7][lane][0]) = make_float4(E1, K1, Zq, th);
-                    *reinterpret_cast<float2*>(&pend[it & 7][lane][4]) = make_float2(m, my);     // the warp's maxima, until the factors replace them
+                    *reinterpret_cast<float4*>(&pend[it & 15][lane][0]) = make_float4(E1, K1, Zq, th);
+                    *reinterpret_cast<float2*>(&pend[it & 15][lane][4]) = make_float2(m, my);     // the warp's maxima, until the factors replace them
                 }
                 combine_records(E1, Zq, th, m, my, lane);
-                if (lane == 0) {
-                    unsigned char* xr = P.xrec + ((size_t)row * g.C + crank) * kXrecBytes;
-                    st_tagged(xr, E1, g.tag); st_tagged(xr + 8, Zq, g.tag); st_tagged(xr + 16, th, g.tag);
-                    st_tagged(xr + 24, m, g.tag); st_tagged(xr + 32, my, g.tag);
-                    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&pbar[it & 7])) : "memory");
+                {
+                    // five (value, tag) words, one per lane
+                    const float v = lane == 0 ? E1 : (lane == 1 ? Zq : (lane == 2 ? th : (lane == 3 ? m : my)));
+                    if (lane < 5) st_tagged(P.xrec + ((size_t)row * g.C + crank) * kXrecBytes + 8 * lane, v, g.tag);
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&pbar[it & 15]));
             }
             if (it - nb >= 0) finish_row(it - nb);
         }
-    } else if (warp == kSW + 1) {
+    } else if (warp == kWCollect) {
         // ================================ collect warp ==================================================
         // Per row: gather the C records of the row from global memory, leave the row scalars and every
         // warp's factors in shared memory for the second visits.
@@ -650,7 +801,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
 #pragma unroll
                     for (int k = 0; k < 5; ++k) ok = ok && (uint32_t)(w[k] >> 32) == g.tag;
                     if (ok) break;
-                    if (++spins > kSpinLimit || ld_volatile_s32(&fail)) { atomicExch(&fail, 1); break; }
+                    if (++spins > spin_limit || ld_volatile_s32(&fail)) { atomicExch(&fail, 1); break; }
+                    __nanosleep(20);
                 }
                 E1 = __uint_as_float((uint32_t)w[0]); Zq = __uint_as_float((uint32_t)w[1]); th = __uint_as_float((uint32_t)w[2]);
                 m = __uint_as_float((uint32_t)w[3]); my = __uint_as_float((uint32_t)w[4]);
@@ -658,26 +810,20 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             combine_records(E1, Zq, th, m, my, lane);
             const float inv_zp = 1.f / E1, inv_zq = 1.f / Zq;
             const float theta = th * inv_zp * inv_zq;
-            mbar_wait<100>(smem_u32(&pbar[it & 7]), (uint32_t)((it >> 3) & 1), &fail);     // this CTA's own record of the row is parked
+            mbar_wait(smem_u32(&pbar[it & 15]), (uint32_t)((it >> 4) & 1), &fail, spin_limit);     // this CTA's own record of the row is parked
             if (lane < kSW) {
-                const float2 mw = *reinterpret_cast<const float2*>(&pend[it & 7][lane][4]);
+                const float2 mw = *reinterpret_cast<const float2*>(&pend[it & 15][lane][4]);
                 float2 f;
                 f.x = (mw.x > -INFINITY ? ex2((mw.x - m) * kLog2e) : 0.f) * inv_zp;
                 f.y = (KIND == RDK_LOGITS ? (mw.y > -INFINITY ? ex2((mw.y - my) * kLog2e) : 0.f) : 1.f) * inv_zq;
                 fzy[pc][lane] = f;
-                *reinterpret_cast<float4*>(&pend[it & 7][lane][4]) = make_float4(f.x, f.y, theta, 0.f);
+                // lanes 0..3 also carry the row scalars the draws need: -m log2e, 1/Zp, -my log2e, 1/Zq
+                const float sc = lane == 0 ? -m * kLog2e : (lane == 1 ? inv_zp : (lane == 2 ? (KIND == RDK_LOGITS ? -my * kLog2e : 0.f) : inv_zq));
+                *reinterpret_cast<float4*>(&pend[it & 15][lane][4]) = make_float4(f.x, f.y, theta, sc);
             }
-            if (lane == 0) {
-                float* sc = scal[pc];
-                sc[0] = -m * kLog2e; sc[1] = inv_zp; sc[2] = KIND == RDK_LOGITS ? -my * kLog2e : 0.f; sc[3] = inv_zq; sc[4] = theta;
-                if (crank == 0) {
-                    float* rec = P.rec + row * kRecFloats;
-                    rec[kRecOffg] = sc[0]; rec[kRecInvZp] = inv_zp; rec[kRecYoffg] = sc[2]; rec[kRecInvZq] = inv_zq;
-                    rec[kRecTheta] = theta; rec[kRecInvN] = inv_n; rec[kRecInvS] = 1.f; rec[kRecS] = 1.f;
-                }
-            }
+            if (lane == 0) scal[pc][4] = theta;
             __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rbar[pc])) : "memory");
+            if (lane == 0) mbar_arrive(smem_u32(&rbar[pc]));
             if (crank == 0 && P.counters && row % P.positions == 0)
                 for (int t = lane; t < P.trials; t += 32) P.counters[(row / P.positions) * P.trials + t] = 0;
         }
@@ -689,18 +835,20 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
         const int lenc_v = lenc & ~(kZPer - 1);
         const uint32_t zbytes = (uint32_t)lenc_v * (uint32_t)sizeof(TZ);
-        const uint32_t kbytes = lane < kSW ? (uint32_t)si.kcs * (uint32_t)sizeof(TY) : 0u;
+        const int l_kcs = min(sd.y, g.ycap);
+        const uint32_t kbytes = lane < kSW ? (uint32_t)l_kcs * (uint32_t)sizeof(TY) : 0u;
         const uintptr_t y_end16 = reinterpret_cast<uintptr_t>(static_cast<const TY*>(P.drafter) +
                                                               (long long)(P.rows - 1) * P.drafter_stride + P.n) & ~uintptr_t(15);
         const long long zstep = (long long)g.G * P.target_stride, ystep = (long long)g.G * P.drafter_stride;
         const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0c;
-        const TY* ny = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + si.r0;
+        const TY* ny = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + sd.x;
         const uint32_t yw_off = zslice + 16u + (uint32_t)(lane & (kSW - 1)) * (uint32_t)g.ystage;
         int s = 0;
         uint32_t eph = 1, st_a = dsm_a, fb = full_a, eb = empty_a;    // a fresh stage counts as released
         unsigned char* st_p = dsm;
         for (int it = 0; it < rows_g; ++it) {
-            mbar_wait<500>(eb, eph, &fail);
+            mbar_wait(eb, eph, &fail, spin_limit);
+            const bool z_issued = it < pre_rows;          // the target slice of this row is on its way already
             // the few elements a 16-byte copy cannot cover go by plain stores: a slice that ends inside a
             // vector, and the very end of the drafter buffer
             const uintptr_t b0 = reinterpret_cast<uintptr_t>(ny), b1 = b0 + kbytes;
@@ -714,12 +862,12 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
                 const int nt = (int)((b1 - t0) / sizeof(TY));
                 for (int k = 0; k < nt; ++k) reinterpret_cast<TY*>(st_p + yw_off + (t0 - a0))[k] = reinterpret_cast<const TY*>(t0)[k];
             }
-            const uint32_t total = zbytes + __reduce_add_sync(0xffffffffu, ybytes);
+            const uint32_t total = (z_issued ? 0u : zbytes) + __reduce_add_sync(0xffffffffu, ybytes);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage was last touched by plain loads and stores
             if (lane == 0) {
                 if (total == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(fb) : "memory");
                 else asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(total) : "memory");
-                for (uint32_t off = 0; off < zbytes; off += 32768u) {
+                for (uint32_t off = 0; !z_issued && off < zbytes; off += 32768u) {
                     const uint32_t sz = min(32768u, zbytes - off);
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                                  ::"r"(st_a + off), "l"(reinterpret_cast<const char*>(nz) + off), "r"(sz), "r"(fb) : "memory");
@@ -733,61 +881,37 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             st_a += stage; st_p += stage; fb += 8u; eb += 8u;
             if (++s == g.NS) { s = 0; eph ^= 1u; st_a = dsm_a; st_p = dsm; fb = full_a; eb = empty_a; }
         }
+        if (ld_volatile_s32(&fail)) {
+            // A wait gave up somewhere, so nobody may have waited for the last copies: let them land before
+            // the CTA leaves (bounded as well, on a count of its own).
+            for (int k = 0; k < g.NS && k < rows_g; ++k) {
+                const int last_it = ((rows_g - 1 - k) / g.NS) * g.NS + k;        // last row that used stage k
+                const uint32_t bar = full_a + 8u * (uint32_t)k, parity = (uint32_t)((last_it / g.NS) & 1);
+                uint32_t done = 0;
+                for (unsigned spins = 0; !done && spins < (1u << 16); ++spins) {
+                    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+                    if (!done) __nanosleep(100);
+                }
+            }
+        }
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (kTmem && warp == 0) {               // every path ends here, also after a wait that gave up
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base_s), "r"(kTmemCols) : "memory");
+    }
     if (tid == 0 && fail && P.status_word) atomicCAS(P.status_word, 0, (int)RDK_ERR_TIMEOUT);
 }
 
-// ------------------------------------------------------------------------------------------------
-// kernel 2
-// ------------------------------------------------------------------------------------------------
-struct DrawCtx {
-    const void* zrow; const void* yrow; bool zvec;
-    const uint32_t* mask; const int32_t* rank;
-    int N;
-    Scal c;
-};
-
-// p and w of the 8 tokens starting at global token jb (a multiple of 8)
-template <typename TZ, typename TY, int KIND>
-__device__ __forceinline__ void draw_pw(const DrawCtx& d, int jb, float (&p)[kVec], float (&w)[kVec]) {
-    float z[kVec];
-    load8<TZ>(static_cast<const TZ*>(d.zrow), jb, d.N, d.zvec, -INFINITY, z);
-    const uint32_t word = __ldg(d.mask + (jb >> 5));
-    const int rbase = __ldg(d.rank + (jb >> 5));          // issued together with the mask and the logits
-    const int sh = jb & 31;
-    const uint32_t mb = (word >> sh) & 0xffu;
-#pragma unroll
-    for (int k = 0; k < kVec; ++k) {
-        p[k] = ex2(fmaf(z[k], kLog2e, d.c.offg)) * d.c.inv_zp;
-        w[k] = taylor_w(d.c, p[k], 0.f);
-    }
-    if (!mb) return;
-    int r = rbase + __popc(word & ((1u << sh) - 1u));
-#pragma unroll
-    for (int k = 0; k < kVec; ++k) {
-        if (mb & (1u << k)) {
-            const float y = to_float<TY>(static_cast<const TY*>(d.yrow)[r]);     // ascending kept ids: rank = drafter index
-            ++r;
-            const float qp = (KIND == RDK_LOGITS ? ex2(fmaf(y, kLog2e, d.c.yoffg)) : y) * d.c.inv_zq;
-            w[k] = taylor_w(d.c, p[k], qp);
-        }
-    }
+__device__ __forceinline__ bool index_matches(const RowParams& P) {
+    return P.header[kHdrMagic] == kIdxMagic && P.header[kHdrN] == P.N && P.header[kHdrn] == P.n;
 }
 
-enum { kPickW = 0, kPickR = 1, kPickP = 2 };
-
-template <typename TZ, typename TY, int KIND>
-__device__ __forceinline__ void draw_x(const DrawCtx& d, int what, int jb, int seg_end, float (&p)[kVec], float (&w)[kVec], float (&x)[kVec]) {
-#pragma unroll
-    for (int k = 0; k < kVec; ++k) { p[k] = 0.f; w[k] = 0.f; x[k] = 0.f; }
-    if (jb >= seg_end) return;
-    draw_pw<TZ, TY, KIND>(d, jb, p, w);
-#pragma unroll
-    for (int k = 0; k < kVec; ++k)
-        x[k] = what == kPickW ? w[k] : (what == kPickR ? fmaxf(0.f, p[k] - w[k] * d.c.inv_s) : p[k]);
-}
-
+// ------------------------------------------------------------------------------------------------
+// kernel 2: one CTA per (row, trial) turns the row's record into draws
+// ------------------------------------------------------------------------------------------------
 // DT threads per CTA: half of the warps work on the draft draw, half on the residual draw.
 template <typename TZ, typename TY, int KIND, int DT>
 __global__ void __launch_bounds__(DT)
@@ -802,14 +926,15 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
     const int row = blockIdx.x / P.trials, t = blockIdx.x % P.trials;
     const float* rec = P.rec + (long long)row * kRecFloats;
     DrawCtx d;
-    const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
-    const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
     if (!index_matches(P)) return;                 // kernel 1 has reported it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a following stream kernel may set itself up meanwhile
-    asm volatile("griddepcontrol.wait;" ::: "memory");   // kernel 1 (launched just before) is complete and visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // kernel 1 (launched just before) is complete and visible; so is
+                                                         // whatever produced this call's inputs
+    const float* u = P.uniforms + ((long long)row * P.trials + t) * 4;
+    const float u0 = __ldg(u), u1 = __ldg(u + 1), u2 = __ldg(u + 2);
     d.c.offg = __ldcg(rec + kRecOffg); d.c.inv_zp = __ldcg(rec + kRecInvZp); d.c.yoffg = __ldcg(rec + kRecYoffg);
-    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = __ldcg(rec + kRecInvN);
-    d.c.inv_s = __ldcg(rec + kRecInvS);
+    d.c.inv_zq = __ldcg(rec + kRecInvZq); d.c.theta = __ldcg(rec + kRecTheta); d.c.inv_n = 1.f / (float)P.N;
+    d.c.inv_s = 1.f;
 
     if (warp < 3) {   // fp64 prefix sums over the segments: warp 0 those of w, warp 1 of max(0, p - q~), warp 2 of p
         double* cdf = warp == 0 ? cdfW : (warp == 1 ? cdfR : cdfP);
@@ -862,8 +987,8 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
     const int seg_lo = (int)min((long long)seg * Lw, (long long)P.N);
     const int seg_end = (int)min((long long)P.N, (long long)seg_lo + Lw);
     const int nch = (Lw + kSeg - 1) / kSeg;
+    float p[kVec], w[kVec], x[kVec];          // of the last chunk this warp summed
     for (int ch = wg; ch < nch; ch += kGW) {
-        float p[kVec], w[kVec], x[kVec];
         draw_x<TZ, TY, KIND>(d, what, seg_lo + ch * kSeg + lane * kVec, seg_end, p, w, x);
         float s = 0.f;
 #pragma unroll
@@ -888,8 +1013,8 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
         if (chosen < 0) {
             if (wg == 0 && lane == 0) { res_tok[g] = seg_lo; res_p[g] = 0.f; res_w[g] = 0.f; }
         } else if (chosen % kGW == wg) {
-            float p[kVec], w[kVec], x[kVec];
-            draw_x<TZ, TY, KIND>(d, what, seg_lo + chosen * kSeg + lane * kVec, seg_end, p, w, x);
+            // the chunk is still in this warp's registers unless the warp went on to a later one
+            if (chosen + kGW < nch) draw_x<TZ, TY, KIND>(d, what, seg_lo + chosen * kSeg + lane * kVec, seg_end, p, w, x);
             int sel = pick_in_segment(x, r_in, lane);
             if (sel < 0) sel = 0;
             float ps = 0.f, ws = 0.f;
@@ -934,48 +1059,67 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-static size_t stream_smem(const StreamGeo& g, size_t es) {
-    const size_t stage = (size_t)kSW * g.Lw * es + 16 + (size_t)kSW * g.ystage;
-    return (size_t)g.NS * stage + (size_t)kSW * g.ycap * (8 * g.NB + 2) + (size_t)g.NS * 16;   // + cache (8 bytes per live row) and offsets (2 bytes) per slot, barriers
+static int fast_steps(const StreamGeo& g, int nit) {
+    const int nst = g.ycap / 64;
+    return (nit == kFastNit && nst >= 1 && nst <= kMaxFastSteps) ? nst : 0;
 }
 
-// Group size, segment length, stage count and cache capacity for a vocabulary of N tokens with n
-// kept ids; false when the shapes do not fit shared memory.
-static bool plan_stream(int N, int n, size_t es, size_t ys, StreamGeo& g) {
-    const size_t budget = 218 * 1024;      // dynamic shared memory a CTA may ask for, less the static part (about 9 KB)
-    const int vt = 32 * (int)(16 / es);    // tokens one warp covers with one 16-byte vector per lane
-    int C = (N + kSW * 4 * vt - 1) / (kSW * 4 * vt);
-    if (C > kMaxGroup) C = kMaxGroup;
-    g.nv = (N + C * kSW * vt - 1) / (C * kSW * vt);
-    g.Lw = g.nv * vt;
-    g.C = (N + kSW * g.Lw - 1) / (kSW * g.Lw);          // no CTA of a group without tokens
-    if ((g.Lw + kSeg - 1) / kSeg > kMaxChunks || (size_t)kSW * g.Lw * es + 16 > 65535) return false;   // slice offsets are 16-bit
+// offsets_in_smem = false is the unrolled route: offsets in registers and the pair cache in tensor memory
+static size_t stream_smem(const StreamGeo& g, size_t es, bool offsets_in_smem) {
+    const size_t stage = (size_t)kSW * g.Lw * es + 16 + (size_t)kSW * g.ystage;
+    // + cache (8 bytes per slot and live row) and offsets (2 bytes per slot) where they live here, barriers
+    return (size_t)g.NS * stage + (offsets_in_smem ? (size_t)kSW * g.ycap * (8 * g.NB + 2) : 0) + (size_t)g.NS * 16;
+}
+
+// Stage count, live rows and cache capacity for a vocabulary of N tokens with n kept ids; false when
+// the shapes do not fit shared memory.
+static bool plan_stream(int N, int n, size_t es, size_t ys, bool fast_types, StreamGeo& g) {
+    const size_t budget = 212 * 1024;      // dynamic shared memory a CTA may ask for: 227 KB less the static part (14.2 KB)
+    StreamSegs sg;
+    if (!stream_segments(N, es, sg)) return false;
+    g.C = sg.C; g.Lw = sg.Lw; g.nv = sg.nv;
+    if ((g.Lw + kSeg - 1) / kSeg > kMaxChunks) return false;
     const long long expect = ((long long)n * g.Lw + N - 1) / N;
     long long cap = expect + expect / 8 + 32;
     const long long most = (long long)(n < g.Lw ? n : g.Lw) + 1;
     if (cap > most) cap = most;
     cap = (cap + 63) / 64 * 64;
-    // The exchange of a row between the CTAs of its group takes about as long as two first visits, so
-    // the second visit should trail by several rows: prefer live rows over stages, then give up cache.
+    auto fits = [&](long long c) {
+        g.ycap = (int)c;
+        g.ystage = (int)((((size_t)c + 16) * ys + 15) & ~size_t(15));
+        const bool in_regs = fast_types && fast_steps(g, g.nv) > 0;
+        return stream_smem(g, es, !in_regs) <= budget;
+    };
+    // The exchange of a row between the CTAs of its group takes several microseconds (two round trips to L2
+    // and the folding on either side), and a row holds its place in the pair cache for that long: the
+    // second visit should trail by as many rows as there is room for.
+    // Unrolled route: the pair cache is in tensor memory (128 columns per warp, 4 per step and live row), and
+    // shared memory goes to the stages, of which more than the HBM latency needs are of no use.
+    g.ycap = (int)cap;
+    if (fast_types && fast_steps(g, g.nv) > 0) {
+        const int nst = fast_steps(g, g.nv);
+        g.NB = kTmemWarpCols / (4 * nst);
+        if (g.NB > kMaxNB) g.NB = kMaxNB;
+        for (g.NS = 4; g.NS >= 2; --g.NS)
+            if (fits(cap)) return true;
+    }
+    // Otherwise the cache shares shared memory with the stages: prefer live rows over stages, then give up cache.
     static const int pref[][2] = {{4, 3}, {5, 2}, {4, 2}, {3, 3}, {3, 2}};     // {NB, NS}, by measured speed
     for (const auto& pr : pref) {
         g.NB = pr[0]; g.NS = pr[1];
-        g.ycap = (int)cap;
-        g.ystage = (int)((((size_t)cap + 16) * ys + 15) & ~size_t(15));
-        if (stream_smem(g, es) <= budget) return true;
+        if (fits(cap)) return true;
     }
-    for (long long c = cap - 64; c >= 64; c -= 64) {
-        g.ycap = (int)c;
-        g.ystage = (int)((((size_t)c + 16) * ys + 15) & ~size_t(15));
-        if (stream_smem(g, es) <= budget) return true;
-    }
+    for (long long c = cap - 64; c >= 64; c -= 64)
+        if (fits(c)) return true;
     return false;
 }
 
-template <typename TZ, typename TY, int KIND, int NIT>
+static std::atomic<unsigned> g_spin_limit{kSpinLimitDefault};
+
+template <typename TZ, typename TY, int KIND, int NIT, int NST>
 static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s) {
-    auto kern = rdk_stream_kernel<TZ, TY, KIND, NIT>;
-    const size_t smem = stream_smem(g, sizeof(TZ));
+    auto kern = rdk_stream_kernel<TZ, TY, KIND, NIT, NST>;
+    const size_t smem = stream_smem(g, sizeof(TZ), NST == 0);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // how many CTAs are resident at once (cached per kernel instance, shared-memory size and device)
@@ -1004,17 +1148,18 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;      // the CTAs of a group wait for one another: all must be resident
     attr[0].val.cooperative = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set itself up while an earlier call's draw kernel drains
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set itself up while the previous kernel drains
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static thread_local int c_pdl = 1;                // whether the two attributes are accepted together on this system
-    cfg.numAttrs = c_pdl ? 2 : 1;
+    static std::atomic<int> c_pdl{1};                 // whether the two attributes are accepted together on this system
+    const int with_pdl = c_pdl.load();
+    cfg.numAttrs = with_pdl ? 2 : 1;
     e = cudaLaunchKernelEx(&cfg, kern, P, g);
-    if (e != cudaSuccess && c_pdl) {
+    if (with_pdl && (e == cudaErrorNotSupported || e == cudaErrorInvalidValue)) {
         (void)cudaGetLastError();
-        c_pdl = 0;
         cfg.numAttrs = 1;
         e = cudaLaunchKernelEx(&cfg, kern, P, g);
+        if (e == cudaSuccess) c_pdl.store(0);         // the pair is what this system refuses
     }
     if (e == cudaErrorCooperativeLaunchTooLarge) {   // fewer SMs at hand than the device reports: the one-CTA-per-row kernel serves
         (void)cudaGetLastError();
@@ -1044,13 +1189,27 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
 template <typename TZ, typename TY, int KIND>
 static cudaError_t launch_nit(const RowParams& P, const StreamGeo& g, cudaStream_t s) {
     // the common segment length (four 16-byte vectors per lane) gets the register-resident sweep
-    if (g.nv == 4) return launch_stream<TZ, TY, KIND, 4>(P, g, s);
-    return launch_stream<TZ, TY, KIND, 0>(P, g, s);
+    if (g.nv == kFastNit) return launch_stream<TZ, TY, KIND, kFastNit, 0>(P, g, s);
+    return launch_stream<TZ, TY, KIND, 0, 0>(P, g, s);
 }
 
 template <typename TZ, typename TY>
 static cudaError_t launch_kind_s(const RowParams& P, int kind, const StreamGeo& g, cudaStream_t s) {
     return kind == RDK_LOGITS ? launch_nit<TZ, TY, RDK_LOGITS>(P, g, s) : launch_nit<TZ, TY, RDK_PROBS>(P, g, s);
+}
+
+// bf16 logits on both sides with the common segment length: the kept-token passes unrolled
+static cudaError_t launch_fast(const RowParams& P, const StreamGeo& g, int nst, cudaStream_t s) {
+    using B = __nv_bfloat16;
+    switch (nst) {
+        case 1: return launch_stream<B, B, RDK_LOGITS, kFastNit, 1>(P, g, s);
+        case 2: return launch_stream<B, B, RDK_LOGITS, kFastNit, 2>(P, g, s);
+        case 3: return launch_stream<B, B, RDK_LOGITS, kFastNit, 3>(P, g, s);
+        case 4: return launch_stream<B, B, RDK_LOGITS, kFastNit, 4>(P, g, s);
+        case 5: return launch_stream<B, B, RDK_LOGITS, kFastNit, 5>(P, g, s);
+        case 6: return launch_stream<B, B, RDK_LOGITS, kFastNit, 6>(P, g, s);
+        default: return cudaErrorNotSupported;
+    }
 }
 
 static size_t ws_off_counters(int rows) { return idx_align((size_t)rows * kRecFloats * sizeof(float)); }
@@ -1061,7 +1220,7 @@ size_t stream_workspace_bytes(int rows, int batch, int trials) {
 }
 
 // A non-zero 32-bit value that differs from the one of every recent call of this process and that
-// stale memory is unlikely to hold.  (The draw kernel wipes a call's records, so a captured call that
+// stale memory is unlikely to hold.  (The kernel wipes a call's records, so a captured call that
 // is replayed with this same value starts from a workspace without them.)
 static uint32_t next_tag() {
     static std::atomic<uint32_t> ctr{
@@ -1070,23 +1229,46 @@ static uint32_t next_tag() {
     return t ? t : 0x9E3779B9u;
 }
 
+static bool fast_types(int tz, int ty, int kind) { return tz == RDK_BF16 && ty == RDK_BF16 && kind == RDK_LOGITS; }
+
+const char* stream_ineligible(const RowParams& P, int tz, int ty, int kind, int batch, const void* ws, size_t ws_bytes) {
+    const size_t es = tz == RDK_F32 ? 4 : 2, ys = ty == RDK_F32 ? 4 : 2;
+    if (P.N < kStreamMinN) return "N < 4096";
+    if (P.qtilde) return "q~ is written out";
+    if (P.rows <= 0 || P.trials <= 0) return "no draws";
+    if (P.prior) return "separate prior";
+    // rows of the target start on 16-byte boundaries; drafter values are read in aligned pairs
+    if ((reinterpret_cast<uintptr_t>(P.target) & 15u) || ((P.target_stride * (long long)es) & 15)) return "target rows not 16-byte aligned";
+    if ((reinterpret_cast<uintptr_t>(P.drafter) & 15u) || (P.drafter_stride & 1)) return "drafter base not 16-byte aligned or odd drafter row stride";
+    if ((long long)P.rows * P.trials > 0x7fffffffLL) return "too many draws";
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < stream_workspace_bytes(P.rows, batch, P.trials)) return "no workspace";
+    // ascending, valid kept ids only, as recorded when the index was built (the kernel re-checks the header)
+    if (index_order(P.header, P.N, P.n) != 1) return "kept ids not ascending and valid (or index not prepared at this address)";
+    StreamGeo g;
+    if (!plan_stream(P.N, P.n, es, ys, fast_types(tz, ty, kind), g)) return "shapes beyond shared memory";
+    return nullptr;
+}
+
+void set_stream_spin_limit(unsigned limit) { g_spin_limit.store(limit ? limit : kSpinLimitDefault); }
+
 cudaError_t launch_stream_linear(RowParams P, int tz, int ty, int kind, int batch, void* ws, size_t ws_bytes, cudaStream_t s) {
     const size_t es = tz == RDK_F32 ? 4 : 2, ys = ty == RDK_F32 ? 4 : 2;
-    if (P.N < kMinStreamN || P.qtilde || P.rows <= 0 || P.trials <= 0 || !ws) return cudaErrorNotSupported;
-    // rows of the target start on 16-byte boundaries; drafter values are read in aligned pairs
-    if ((reinterpret_cast<uintptr_t>(P.target) & 15u) || ((P.target_stride * (long long)es) & 15)) return cudaErrorNotSupported;
-    if ((reinterpret_cast<uintptr_t>(P.drafter) & 15u) || (P.drafter_stride & 1)) return cudaErrorNotSupported;
-    if ((long long)P.rows * P.trials > 0x7fffffffLL) return cudaErrorNotSupported;
-    if ((reinterpret_cast<uintptr_t>(ws) & 15u) || ws_bytes < stream_workspace_bytes(P.rows, batch, P.trials)) return cudaErrorNotSupported;
-    // ascending, valid kept ids only, as recorded when the index was built (kernel 1 re-checks the header)
-    if (index_order(P.header, P.N, P.n) != 1) return cudaErrorNotSupported;
+    if (stream_ineligible(P, tz, ty, kind, batch, ws, ws_bytes)) return cudaErrorNotSupported;
     StreamGeo g;
-    if (!plan_stream(P.N, P.n, es, ys, g)) return cudaErrorNotSupported;
+    if (!plan_stream(P.N, P.n, es, ys, fast_types(tz, ty, kind), g)) return cudaErrorNotSupported;
     g.G = 0;
     g.tag = next_tag();
+    g.spin_limit = g_spin_limit.load();
+    const KeptIndexView v = make_view(P.header, P.N, P.n);
+    g.segdesc = v.segdesc[es == 2 ? 0 : 1];
+    g.goff = v.goff[es == 2 ? 0 : 1];
     P.rec = static_cast<float*>(ws);
     P.counters = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + ws_off_counters(P.rows));
     P.xrec = reinterpret_cast<unsigned char*>(ws) + ws_off_xrec(P.rows, batch, P.trials);
+    if (fast_types(tz, ty, kind)) {
+        const int nst = fast_steps(g, g.nv);
+        if (nst > 0) return launch_fast(P, g, nst, s);
+    }
     if (tz == RDK_F32) return ty == RDK_F32 ? launch_kind_s<float, float>(P, kind, g, s) : launch_kind_s<float, __nv_bfloat16>(P, kind, g, s);
     return ty == RDK_F32 ? launch_kind_s<__nv_bfloat16, float>(P, kind, g, s) : launch_kind_s<__nv_bfloat16, __nv_bfloat16>(P, kind, g, s);
 }
@@ -1101,12 +1283,13 @@ extern "C" int rdk_stream_geometry(int32_t N, int32_t n, int32_t target_dtype, i
         return RDK_ERR_INVALID_ARG;
     }
     const size_t es = target_dtype == RDK_F32 ? 4 : 2, ys = drafter_dtype == RDK_F32 ? 4 : 2;
+    const bool ft = fast_types(target_dtype, drafter_dtype, RDK_LOGITS);
     StreamGeo g;
     *out = rdk_stream_geometry_t{};
-    out->supported = N >= kMinStreamN && plan_stream(N, n, es, ys, g) ? 1 : 0;
+    out->supported = plan_stream(N, n, es, ys, ft, g) ? 1 : 0;
     if (!out->supported) return RDK_OK;
     out->ctas_per_row = g.C; out->warps_per_cta = kSW; out->segment_tokens = g.Lw; out->stages = g.NS;
     out->live_rows = g.NB; out->cached_slots_per_warp = g.ycap;
-    out->dynamic_shared_bytes = (int64_t)stream_smem(g, es);
+    out->dynamic_shared_bytes = (int64_t)stream_smem(g, es, !(ft && fast_steps(g, g.nv) > 0));
     return RDK_OK;
 }
