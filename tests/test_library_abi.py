@@ -94,6 +94,28 @@ def test_argument_errors_are_reported_on_the_host(B):
     assert st == B.RDK_ERR_WORKSPACE_TOO_SMALL
 
 
+def test_route_query_reports_host_side_argument_errors(B):
+    L = B.lib()
+    pb = B.rdk_problem()
+    pb.N, pb.n, pb.batch, pb.positions = 0, 4, 1, 1
+    why = C.c_char_p()
+    assert L.rdk_sample_route(C.byref(pb), 0, None, None, 1, None, 0, C.byref(why)) == -B.RDK_ERR_INVALID_ARG
+    pb.N, pb.kept_index = 8192, 256
+    pb.target_dtype = pb.drafter_dtype = B.RDK_BF16
+    # a precomputed w never streams; nor does a problem whose flags ask for the row kernel
+    assert L.rdk_sample_route(C.byref(pb), 1, None, None, 1, None, 0, C.byref(why)) == B.RDK_ROUTE_ROW_KERNEL
+    pb.flags = B.RDK_FLAG_ROW_KERNEL
+    assert L.rdk_sample_route(C.byref(pb), 0, None, None, 1, None, 0, C.byref(why)) == B.RDK_ROUTE_ROW_KERNEL
+    assert b"RDK_FLAG_ROW_KERNEL" in why.value
+    pb.flags = 2
+    assert L.rdk_sample_route(C.byref(pb), 0, None, None, 1, None, 0, None) == -B.RDK_ERR_INVALID_ARG
+    # an index this process never prepared at that address: not known to be ascending
+    pb.flags = 0
+    dummy = C.c_void_p(4096)
+    assert L.rdk_sample_route(C.byref(pb), 0, dummy, dummy, 1, dummy, 1 << 30, C.byref(why)) == B.RDK_ROUTE_ROW_KERNEL
+    assert b"kept ids" in why.value
+
+
 def test_binding_refuses_wrong_tensor_types(B):
     import torch
     with pytest.raises(TypeError):
@@ -119,10 +141,13 @@ def test_stream_geometry_covers_the_vocabulary_and_fits_shared_memory(B):
             segs = g["ctas_per_row"] * g["warps_per_cta"]
             assert segs * g["segment_tokens"] >= N and segs <= 256 and 1 <= g["ctas_per_row"] <= 16
             assert (segs - g["warps_per_cta"]) * g["segment_tokens"] < N            # the last CTA is not idle
-            assert 2 <= g["stages"] <= 3 and 3 <= g["live_rows"] <= 5
+            assert 2 <= g["stages"] <= 4 and 3 <= g["live_rows"] <= 8
             assert g["cached_slots_per_warp"] % 64 == 0 and g["cached_slots_per_warp"] >= 64
-            assert g["dynamic_shared_bytes"] <= 218 * 1024
+            assert g["dynamic_shared_bytes"] <= 212 * 1024
     big = rdk.rdk_stream_geometry(128256, 32064)
     assert big["ctas_per_row"] == 8 and big["segment_tokens"] == 1024      # the benchmark shape
+    # bf16 logits with the common segment length keep the pair cache in tensor memory: 128 columns per
+    # warp at 4 per 64-slot step and live row, so shared memory holds stages only
+    assert big["live_rows"] * (big["cached_slots_per_warp"] // 64) * 4 <= 128 and big["stages"] >= 3
     assert rdk.rdk_stream_geometry(1000, 10)["supported"] == 0              # small vocabularies take the row kernel
     assert rdk.rdk_stream_geometry(1 << 21, 1000)["supported"] == 0         # too large for shared memory
