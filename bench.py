@@ -1,12 +1,14 @@
 """Benchmark of the RDK hot path on B200.
 
-One "step" takes one batch of the Llama-3-scale workload (target vocabulary N = 128256, drafter
+One "step" takes one batch of the Llama-3-scale workload C2 (target vocabulary N = 128256, drafter
 keeps n = 32064 ids, 64 sequences x 5 draft positions = 320 rows, bf16 logits) through the whole
 path: drafter/target soft-max, Token-Level Intersection, first-order redistribution, draft draw,
 rejection test, acceptance rate, residual draw and the per-sequence accepted length.  The metric
-is verified draft tokens per second = rows x steps / elapsed.
+is verified draft tokens per second = rows x steps / elapsed.  The same line carries, under
+"workloads", the other sizes of the linear path (C3, C4) against the HBM roofline and the exact
+tensor-core path (C5) against the bf16 tensor peak.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C2|C3|C4|C5]
 
 Prints ONE JSON line.  With --impl reference the CPU checker (oracle/) is timed on the host cores
 instead; that arm touches no GPU.
@@ -16,6 +18,7 @@ from __future__ import annotations
 import argparse
 import hashlib
 import json
+import math
 import os
 import sys
 import threading
@@ -25,15 +28,16 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-WORKLOAD = "C2"              # default: the configuration the metric is quoted on (--workload picks another)
+WORKLOAD = "C2"              # the configuration the metric is quoted on (--workload picks another as the headline)
+OTHER_WORKLOADS = ("C3", "C4", "C5")
 N_BUFFER_SETS = 6            # distinct input batches rotated through, so every step reads HBM
 METRIC = "verified draft tokens/sec"
 UNIT = "tokens/s"
+MIN_TIMED_SECONDS = 0.5      # the K-step loop is repeated until at least this much has been timed (and 5 times)
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "368495009f2b0618217eb5ae984b3a808be9932e751962e2c1759995890eed39",
-               "bytes_per_launch": 102941952 + 3496704}   # rdk_stream_kernel, profiles/rdk_stream_and_draw_kernels_C2.md
+NCU_TRAFFIC = {"sources_sha256": "", "bytes_per_launch": {}}
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 
@@ -45,13 +49,15 @@ def _kernel_sources_hash() -> str:
     return h.hexdigest()
 
 
-def _peaks():
+def _measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return {"hbm": float(d["hbm_gbs"]), "tensor": float(d["bf16_tflops"]), "tensor_sustained": float(d["bf16_tflops_sustained"]),
+                "source": "measured (MEASURED_PEAKS.json: hbm_gbs, bf16_tflops burst, bf16_tflops_sustained)"}
+    return {"hbm": 6650.0, "tensor": 1590.0, "tensor_sustained": 1400.0,
+            "source": "fallback (6.65 TB/s, 1.59 / 1.4 PFLOP/s: earlier measurements on this pool)"}
 
 
 class ClockSampler(threading.Thread):
@@ -109,6 +115,7 @@ class ClockSampler(threading.Thread):
 
     def stop(self):
         self._stop_evt.set()
+        self.join(timeout=1.0)
 
     def summary(self):
         if not self.ok or not self.samples:
@@ -118,7 +125,10 @@ class ClockSampler(threading.Thread):
                 "samples": len(s)}
 
 
-def _cpu_baseline(cfg, min_seconds: float = 10.0, pool_rows: int = 64):
+# ----------------------------------------------------------------------------------------------
+# the CPU checker as a timed baseline (the one place besides --impl reference where oracle/ runs)
+# ----------------------------------------------------------------------------------------------
+def _cpu_baseline_linear(cfg, name: str, min_seconds: float = 10.0, pool_rows: int = 64):
     """Time the CPU checker, as it stands, on rows of the same workload for about min_seconds."""
     import numpy as np
 
@@ -138,7 +148,41 @@ def _cpu_baseline(cfg, min_seconds: float = 10.0, pool_rows: int = 64):
         dt = time.perf_counter() - t0
         if dt >= min_seconds:
             break
-    return done / dt, dt, done
+    return {"value": done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{done} rows of {name} through oracle.rdk_row (float64 numpy, one thread, {dt:.1f} s)"}
+
+
+def _cpu_baseline_exact(cfg, name: str, rows: int = 256, cols: int = 4096):
+    """The checker's exact path on a bounded sample: `rows` rows, the contraction on `cols` seeded columns of
+    the affinity matrix (built by the checker beforehand, untimed like the library's preprocessing) and scaled to
+    all N columns, plus the checker's sampling step on a weight vector of full length."""
+    import numpy as np
+
+    import workloads as W
+    from oracle import rdk_oracle as O
+    inp = W.make_inputs(cfg.with_rows(rows, 1), device="cpu", with_embeddings=True)
+    kappa = inp["kept_ids"].numpy()
+    rng = np.random.default_rng(cfg.seed)
+    sel = np.sort(rng.choice(cfg.N, cols, replace=False))
+    Mcols = O.round_to_bf16(O.affinity_columns(W.to_f64(inp["embeddings"]), kappa, cfg.tau, sel))
+    z = [W.to_f64(inp["target"][r]) for r in range(rows)]
+    y = [W.to_f64(inp["drafter"][r]) for r in range(rows)]
+    u = inp["uniforms"].numpy().astype(np.float64)
+    t0 = time.perf_counter()
+    wc = []
+    for r in range(rows):
+        qk = O.round_to_bf16(O.drafter_qprime(y[r], kappa, cfg.N, cfg.drafter_kind)[kappa])
+        wc.append(O.redistribute_exact(qk, Mcols))
+    t_contract = (time.perf_counter() - t0) * (cfg.N / cols)
+    t0 = time.perf_counter()
+    for r in range(rows):
+        O.rdk_row(z[r], None, kappa, u[r], "given", w_given=np.tile(wc[r], cfg.N // cols))
+    t_sample = time.perf_counter() - t0
+    dt = t_contract + t_sample
+    return {"value": rows / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": (f"{rows} rows of {name}: oracle.redistribute_exact on {cols} of {cfg.N} seeded columns of the checker's "
+                       f"bf16-rounded affinity matrix, time scaled by {cfg.N // cols} ({t_contract:.1f} s), plus oracle.rdk_row "
+                       f"(mode 'given') on full-length weights ({t_sample:.1f} s); float64 numpy, one thread")}
 
 
 def run_reference(args):
@@ -203,13 +247,263 @@ def whole_job_value(rows_per_rank: int, trials: int, steps: int, world: int, ms:
     return world * rows_per_rank * trials * steps / (ms * 1e-3)
 
 
-def _peak_tensor():
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(path):
-        with open(path) as f:
-            d = json.load(f)
-        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
-    return 1590.0, 1400.0, "fallback (1.59 PFLOP/s burst, earlier measurement on this pool)"
+def repeats_for(est_ms_per_step: float, steps: int, min_seconds: float = MIN_TIMED_SECONDS) -> int:
+    """How often the K-step loop is timed: at least five times and until min_seconds have been timed."""
+    per_loop = max(est_ms_per_step * steps * 1e-3, 1e-6)
+    return int(min(2000, max(5, math.ceil(min_seconds / per_loop))))
+
+
+def median_and_spread(xs):
+    s = sorted(xs)
+    med = s[len(s) // 2] if len(s) % 2 else 0.5 * (s[len(s) // 2 - 1] + s[len(s) // 2])
+    return med, (s[-1] - s[0]) / med if med > 0 else 0.0
+
+
+class Ctx:
+    def __init__(self, torch, B, W, dist, dev, world, rank, local_rank, peaks):
+        self.torch, self.B, self.W, self.dist, self.dev = torch, B, W, dist, dev
+        self.world, self.rank, self.local_rank, self.peaks = world, rank, local_rank, peaks
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+            self.torch.cuda.synchronize()
+
+    def timed(self, fn, n_steps: int) -> float:
+        """Exactly n_steps steps between two events, a barrier and a synchronise on both sides; max over ranks."""
+        t = self.torch
+        e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        self.barrier()
+        e0.record()
+        for i in range(n_steps):
+            fn(i)
+        e1.record()
+        self.barrier()
+        return max_over_ranks(e0.elapsed_time(e1), self.dist, self.dev)
+
+    def timed_repeats(self, fn, n_steps: int, warm_ms: float):
+        reps = repeats_for(warm_ms / max(1, n_steps), n_steps)
+        return [self.timed(fn, n_steps) for _ in range(reps)]
+
+
+def bench_workload(ctx: Ctx, name: str, steps: int, warmup: int, prior: bool, headline: bool, cpu_baseline: bool):
+    """Time one workload; returns the fields of its entry (the headline workload's become the line itself)."""
+    torch, B, W, dev = ctx.torch, ctx.B, ctx.W, ctx.dev
+    cfg = W.CONFIGS[name]
+    exact = cfg.path == "exact"
+    rows, trials = cfg.rows, cfg.trials
+    zb = 2 if cfg.dtype == "bf16" else 4
+    kind = B.RDK_PROBS if cfg.drafter_kind == "probs" else B.RDK_LOGITS
+    row_bytes = cfg.N * zb + cfg.n * zb + trials * 16 + 30
+    # enough distinct batches that one rotation exceeds L2 several times over (C5's operands do so alone)
+    nsets = 1 if exact else max(2, min(N_BUFFER_SETS, int(600e6 // (rows * row_bytes)) + 1))
+    sets = [W.make_inputs(cfg, device=str(dev), variant=v + 100 * ctx.rank, with_embeddings=exact and v == 0)
+            for v in range(nsets)]
+    index = B.rdk_prepare_ids(sets[0]["kept_ids"], cfg.N)
+    outs = [B.alloc_outputs(rows, cfg.batch, trials, dev) for _ in range(nsets)]
+    outs_nolen = [{k: v for k, v in o.items() if k != "accepted_len"} for o in outs]
+    pb = B.make_problem(index, sets[0]["target"], sets[0]["drafter"], cfg.batch, cfg.positions, kind)
+    ws = B.sample_workspace(pb, B.RDK_MODE_LINEAR, trials, dev)
+
+    prep_ms = None
+    kernels = None
+    if exact:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        M = B.rdk_build_affinity(sets[0]["embeddings"], sets[0]["kept_ids"], cfg.tau, B.RDK_AFF_BF16_COLS)
+        e1.record()
+        torch.cuda.synchronize()
+        prep_ms = e0.elapsed_time(e1)
+        w_buf = torch.empty(rows, cfg.N, dtype=torch.float32, device=dev)
+        _, _, ews = B.rdk_redistribute_exact(index, sets[0]["drafter"], M, cfg.batch, cfg.positions, kind, w_out=w_buf)
+
+        def contraction(i):
+            B.rdk_redistribute_exact(index, sets[0]["drafter"], M, cfg.batch, cfg.positions, kind, w_out=w_buf, ws=ews)
+
+        def step(i, out_list=outs):
+            contraction(i)
+            B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, sets[0]["target"], None, w_buf, sets[0]["uniforms"],
+                                    cfg.batch, cfg.positions, kind, out=out_list[0], ws=ws)
+        kernel_fn = contraction
+        launches_per_step = 2 + 2          # operand, contraction; row kernel, accepted length
+        kernels = "exact_operand_kernel + exact_tc_kernel (row sums in its epilogue)"
+    elif prior:
+        # Eq. rdk-taylor with one shared prior row (a static stand-in for the unknown target distribution)
+        shared_prior = sets[-1]["target"][0].clone().contiguous()
+
+        def step(i, out_list=outs):
+            s = sets[i % nsets]
+            B.rdk_sample_and_verify_prior(index, s["target"], shared_prior, s["drafter"], s["uniforms"],
+                                          cfg.batch, cfg.positions, kind, out=out_list[i % nsets])
+        kernel_fn = lambda i: step(i, outs_nolen)
+        launches_per_step = 2              # row kernel, accepted length
+        kernels = "rdk_row_kernel (shared prior)"
+    else:
+        route, why = B.rdk_sample_route(index, B.RDK_MODE_LINEAR, sets[0]["target"], sets[0]["drafter"], cfg.batch,
+                                        cfg.positions, trials, ws, kind)
+        if route != B.RDK_ROUTE_STREAM_KERNEL:
+            raise SystemExit(f"{name}: the benchmark shape would take the one-CTA-per-row kernel ({why}); refusing to time it")
+
+        def step(i, out_list=outs):
+            s = sets[i % nsets]
+            B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, s["target"], s["drafter"], None, s["uniforms"],
+                                    cfg.batch, cfg.positions, kind, out=out_list[i % nsets], ws=ws)
+        kernel_fn = lambda i: step(i, outs_nolen)
+        launches_per_step = 2              # stream kernel, draw kernel
+        kernels = "rdk_stream_kernel + rdk_draw_kernel (route reported by rdk_sample_route)"
+
+    for i in range(max(3, warmup)):
+        step(i)
+    warm_ms = ctx.timed(step, steps)                   # a first, untimed-for-the-record pass sizes the number of repeats
+    sampler = ClockSampler(ctx.local_rank)
+    sampler.start()
+    loop_ms = ctx.timed_repeats(step, steps, warm_ms)
+    # the dominant kernels alone: linear = stream + draw kernels; exact = the contraction call
+    # (operand preparation, tensor-core kernel, row sums)
+    kern_ms = ctx.timed_repeats(kernel_fn, steps, warm_ms)
+    sampler.stop()
+    B.check_status_word(outs[0], f"bench step {name}")
+    ms, spread = median_and_spread(loop_ms)
+    kms, kspread = median_and_spread(kern_ms)
+    kernel_ms = kms / steps
+
+    e2e = None
+    if not prior:
+        e2e_steps = max(3, min(steps, 20))
+        if not exact:
+            # end to end: host (pinned) buffers in, host results out, copies inside the timed region
+            host_sets = [{k: s[k].cpu().pin_memory() for k in ("target", "drafter", "uniforms")} for s in sets[:2]]
+            stage = {"target": torch.empty_like(sets[0]["target"]), "drafter": torch.empty_like(sets[0]["drafter"]),
+                     "uniforms": torch.empty_like(sets[0]["uniforms"]), "ws": ws}
+            host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in outs[0].items() if not k.startswith("_")}
+
+            def e2e_step(i):
+                h = host_sets[i % len(host_sets)]
+                B.rdk_sample_and_verify_host(index, h["target"], h["drafter"], h["uniforms"], cfg.batch, cfg.positions,
+                                             stage, outs[0], host_out, kind)
+            how = "rdk_sample_and_verify_host (pinned host buffers in, host results out)"
+        else:
+            # the exact path has no host entry point of its own: the same two calls a user makes, with the
+            # step's inputs copied in from pinned host memory and the results copied back, all inside the timed region
+            host_in = {k: sets[0][k].cpu().pin_memory() for k in ("target", "drafter", "uniforms")}
+            stage = {k: torch.empty_like(sets[0][k]) for k in host_in}
+            host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in outs[0].items() if not k.startswith("_")}
+
+            def e2e_step(i):
+                for k in stage:
+                    stage[k].copy_(host_in[k], non_blocking=True)
+                B.rdk_redistribute_exact(index, stage["drafter"], M, cfg.batch, cfg.positions, kind, w_out=w_buf, ws=ews)
+                B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, stage["target"], None, w_buf, stage["uniforms"],
+                                        cfg.batch, cfg.positions, kind, out=outs[0], ws=ws)
+                for k, v in host_out.items():
+                    v.copy_(outs[0][k], non_blocking=True)
+                torch.cuda.synchronize()
+            host_sets = [host_in]
+            how = "rdk_redistribute_exact + rdk_sample_and_verify between copies from and to pinned host memory"
+        for i in range(3):
+            e2e_step(i)
+        ms_e2e = ctx.timed(e2e_step, e2e_steps)
+        h2d = sum(host_sets[0][k].numel() * host_sets[0][k].element_size() for k in ("target", "drafter", "uniforms"))
+        d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+        e2e = {"value": ctx.world * rows * trials * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps, "through": how}
+
+    peaks = ctx.peaks
+    if exact:
+        flops = 2.0 * rows * cfg.n * cfg.N
+        achieved = flops / (kernel_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["tensor"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["tensor"], "traffic": None, "kernel_ms": kernel_ms, "flops_per_launch": flops,
+                    "peak_source": peaks["source"], "frac_of_sustained_peak": achieved / peaks["tensor_sustained"],
+                    "tensor_pipe_pct_of_measured_peak": 100.0 * achieved / peaks["tensor"], "kernels": kernels}
+    else:
+        algo_bytes = rows * row_bytes
+        achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
+        traffic = None
+        if not prior and NCU_TRAFFIC["sources_sha256"] == _kernel_sources_hash():
+            traffic = NCU_TRAFFIC["bytes_per_launch"].get(name)
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                    "traffic": traffic, "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": algo_bytes,
+                    "peak_source": peaks["source"], "kernels": kernels}
+
+    cpu = None
+    parity = None
+    if ctx.rank == 0 and cpu_baseline and not prior:
+        cpu = _cpu_baseline_exact(cfg, name) if exact else _cpu_baseline_linear(cfg, name)
+    if ctx.rank == 0 and not exact and not prior:
+        parity = _parity_in_this_run(ctx, cfg, sets[0], outs, index, kind, ws)
+
+    what = ("exact RDK on tensor cores (bf16 affinity, fp32 accumulate) + sampling/verification" if exact
+            else "linear RDK with one shared prior row in Eq. rdk-taylor + sampling/verification" if prior
+            else "linear RDK (first-order redistribution + sampling/verification)")
+    entry = {
+        "value": whole_job_value(rows, trials, steps, ctx.world, ms), "unit": UNIT, "ms_per_step": ms / steps,
+        "timed": {"steps_per_repeat": steps, "repeats": len(loop_ms), "spread": spread, "kernel_repeats": len(kern_ms),
+                  "kernel_spread": kspread, "statistic": "median over repeats of exactly `steps` steps each"},
+        "config": {"workload": f"{name}: {what}, N={cfg.N}, n={cfg.n}, batch={cfg.batch}, "
+                               f"positions={cfg.positions} (rows={rows}), bf16 inputs, trials={trials}",
+                   "rows_per_step": rows, "parallelism": f"replicas x{ctx.world} (no collective)",
+                   "l2": (f"operands of one step ({(cfg.N * cfg.n * 2 + rows * cfg.N * 4) / 1e6:.0f} MB) exceed the 126 MB L2"
+                          if exact else
+                          f"inputs rotate over {nsets} distinct batches ({nsets * rows * row_bytes / 1e6:.0f} MB > 126 MB L2)")},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * steps,
+        "clocks": sampler.summary(), "parity": parity,
+    }
+    if prep_ms is not None:
+        entry["config"]["preprocessing_ms"] = prep_ms
+    del sets, outs, outs_nolen, ws
+    torch.cuda.empty_cache()
+    return entry
+
+
+def _parity_in_this_run(ctx: Ctx, cfg, s0, outs, index, kind, ws, nrows: int = 16):
+    """Rows of this very run recomputed by the CPU checker: how many agree, and how many draws sit on a CDF
+    boundary (counted, not failed).  A handful of rows: the test-suite does the thorough comparison."""
+    import numpy as np
+
+    from oracle import rdk_oracle as O
+    torch, B, W = ctx.torch, ctx.B, ctx.W
+    out = outs[0]
+    B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, s0["target"], s0["drafter"], None, s0["uniforms"], cfg.batch, cfg.positions,
+                            kind, out=out, ws=ws)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(0)
+    rows = sorted(rng.choice(cfg.rows, min(nrows, cfg.rows), replace=False).tolist())
+    kappa = s0["kept_ids"].cpu().numpy()
+    res = {"rows_compared": len(rows), "max_abs_alpha": 0.0, "max_abs_theta": 0.0, "draft_equal": 0, "out_token_equal": 0,
+           "ambiguous_draft": 0, "ambiguous_accept": 0, "ambiguous_residual": 0, "mismatches": 0}
+    d, o, acc = (out[k].cpu().numpy() for k in ("draft_token", "out_token", "accepted"))
+    tol = 1e-5
+    for r in rows:
+        u = s0["uniforms"][r].cpu().numpy().astype(np.float64)
+        ref = O.rdk_row(W.to_f64(s0["target"][r]), W.to_f64(s0["drafter"][r]), kappa, u, "linear", drafter_kind=cfg.drafter_kind)
+        res["max_abs_alpha"] = max(res["max_abs_alpha"], abs(float(out["alpha"][r]) - ref["alpha"]))
+        res["max_abs_theta"] = max(res["max_abs_theta"], abs(float(out["theta"][r]) - ref["theta"]))
+        k = r * cfg.trials
+        S, R = ref["S"], ref["R"]
+        if int(d[k]) == int(ref["draft"][0]):
+            res["draft_equal"] += 1
+        else:
+            t = u[0, 0] * S
+            lo = ref["cdf_w"][int(d[k]) - 1] if d[k] > 0 else 0.0
+            near = min(abs(t - lo), abs(t - ref["cdf_w"][int(d[k])])) <= tol * S
+            res["ambiguous_draft" if near else "mismatches"] += 1
+            continue
+        if bool(acc[k]) != bool(ref["accepted"][0]):
+            p_d, q_d = ref["p"][int(d[k])], ref["qtilde"][int(d[k])]
+            near = abs(u[0, 1] * q_d - p_d) <= tol * max(p_d, q_d)
+            res["ambiguous_accept" if near else "mismatches"] += 1
+            continue
+        if int(o[k]) == int(ref["out_token"][0]):
+            res["out_token_equal"] += 1
+        else:
+            t = u[0, 2] * R
+            lo = ref["cdf_r"][int(o[k]) - 1] if o[k] > 0 else 0.0
+            near = R > 0 and min(abs(t - lo), abs(t - ref["cdf_r"][int(o[k])])) <= tol * R
+            res["ambiguous_residual" if near else "mismatches"] += 1
+    res["note"] = "oracle.rdk_row on seeded rows of this run's first batch; tolerance 1e-5 of the total on CDF boundaries"
+    return res
 
 
 def run_ours(args):
@@ -232,164 +526,41 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-
-    cfg = W.CONFIGS[args.workload]
-    exact = cfg.path == "exact"
-    rows, trials = cfg.rows, cfg.trials
-    zb = 2 if cfg.dtype == "bf16" else 4
-    kind = B.RDK_PROBS if cfg.drafter_kind == "probs" else B.RDK_LOGITS
-    row_bytes = cfg.N * zb + cfg.n * zb + trials * 16 + 30
-    # enough distinct batches that one rotation exceeds L2 several times over (C5's operands do so alone)
-    nsets = 1 if exact else max(2, min(N_BUFFER_SETS, int(600e6 // (rows * row_bytes)) + 1))
-    sets = [W.make_inputs(cfg, device=str(dev), variant=v + 100 * rank, with_embeddings=exact and v == 0)
-            for v in range(nsets)]
-    index = B.rdk_prepare_ids(sets[0]["kept_ids"], cfg.N)
-    outs = [B.alloc_outputs(rows, cfg.batch, trials, dev) for _ in range(nsets)]
-    outs_nolen = [{k: v for k, v in o.items() if k != "accepted_len"} for o in outs]
-    pb = B.make_problem(index, sets[0]["target"], sets[0]["drafter"], cfg.batch, cfg.positions, kind)
-    ws = B.sample_workspace(pb, B.RDK_MODE_LINEAR, trials, dev)
-
-    prep_ms = None
-    if exact:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        M = B.rdk_build_affinity(sets[0]["embeddings"], sets[0]["kept_ids"], cfg.tau, B.RDK_AFF_BF16_COLS)
-        e1.record()
-        torch.cuda.synchronize()
-        prep_ms = e0.elapsed_time(e1)
-        w_buf = torch.empty(rows, cfg.N, dtype=torch.float32, device=dev)
-        _, _, ews = B.rdk_redistribute_exact(index, sets[0]["drafter"], M, cfg.batch, cfg.positions, kind, w_out=w_buf)
-
-        def contraction(i):
-            B.rdk_redistribute_exact(index, sets[0]["drafter"], M, cfg.batch, cfg.positions, kind, w_out=w_buf, ws=ews)
-
-        def step(i, out_list=outs):
-            contraction(i)
-            B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, sets[0]["target"], None, w_buf, sets[0]["uniforms"],
-                                    cfg.batch, cfg.positions, kind, out=out_list[0], ws=ws)
-        launches_per_step = 2 + 2          # operand, contraction; row kernel, accepted length
-    elif args.prior:
-        # Eq. rdk-taylor with one shared prior row (a static stand-in for the unknown target distribution)
-        shared_prior = sets[-1]["target"][0].clone().contiguous()
-
-        def step(i, out_list=outs):
-            s = sets[i % nsets]
-            B.rdk_sample_and_verify_prior(index, s["target"], shared_prior, s["drafter"], s["uniforms"],
-                                          cfg.batch, cfg.positions, kind, out=out_list[i % nsets])
-        launches_per_step = 2              # row kernel, accepted length
-    else:
-        def step(i, out_list=outs):
-            s = sets[i % nsets]
-            B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, s["target"], s["drafter"], None, s["uniforms"],
-                                    cfg.batch, cfg.positions, kind, out=out_list[i % nsets], ws=ws)
-        launches_per_step = 2              # stream kernel, draw kernel
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    def timed(fn, n_steps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        for i in range(n_steps):
-            fn(i)
-        e1.record()
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    ctx = Ctx(torch, B, W, dist, dev, world, rank, local_rank, _measured_peaks())
 
     warmup = max(3, args.warmup)
-    for i in range(warmup):
-        step(i)
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    ms = timed(step, args.steps)
-    # the dominant kernels alone: linear = stream + draw kernels (no accepted length); exact = the
-    # contraction call (operand preparation, tensor-core kernel, row sums)
-    ms_kernel = timed(contraction if exact else (lambda i: step(i, outs_nolen)), args.steps)
-    sampler.stop()
-    sampler.join(timeout=1.0)
-    B.check_status_word(outs[0], "bench step")
-
-    e2e = None
-    if not exact and not args.prior:
-        # end to end: host (pinned) buffers in, host results out, copies inside the timed region
-        e2e_steps = max(3, min(args.steps, 20))
-        host_sets = [{k: s[k].cpu().pin_memory() for k in ("target", "drafter", "uniforms")} for s in sets[:2]]
-        stage = {"target": torch.empty_like(sets[0]["target"]), "drafter": torch.empty_like(sets[0]["drafter"]),
-                 "uniforms": torch.empty_like(sets[0]["uniforms"]), "ws": ws}
-        host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in outs[0].items() if not k.startswith("_")}
-
-        def e2e_step(i):
-            h = host_sets[i % len(host_sets)]
-            B.rdk_sample_and_verify_host(index, h["target"], h["drafter"], h["uniforms"], cfg.batch, cfg.positions,
-                                         stage, outs[0], host_out, kind)
-
-        for i in range(3):
-            e2e_step(i)
-        ms_e2e = timed(e2e_step, e2e_steps)
-        h2d = sum(host_sets[0][k].numel() * host_sets[0][k].element_size() for k in ("target", "drafter", "uniforms"))
-        d2h = sum(v.numel() * v.element_size() for v in host_out.values())
-        e2e = {"value": world * rows * trials * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps}
+    head = bench_workload(ctx, args.workload, args.steps, warmup, args.prior, True, not args.no_cpu_baseline)
+    others = {}
+    if not args.prior and not args.only:
+        for name in OTHER_WORKLOADS:
+            if name == args.workload:
+                continue
+            # the other sizes ride along with fewer steps per repeat (their steps are 4 to 10 times longer)
+            k = max(3, min(args.steps, 100))
+            e = bench_workload(ctx, name, k, 3, False, False, (not args.no_cpu_baseline) and W.CONFIGS[name].path == "exact")
+            others[name] = {"value": e["value"], "unit": e["unit"], "ms_per_step": e["ms_per_step"], "steps": k, "timed": e["timed"],
+                            "kernel_ms": e["roofline"]["kernel_ms"], "roofline": e["roofline"], "clocks": e["clocks"],
+                            "config": e["config"], "gpu_launches": e["gpu_launches"]}
+            if e["cpu_baseline"] is not None:
+                others[name]["cpu_baseline"] = e["cpu_baseline"]
+            if W.CONFIGS[name].path == "exact":
+                others[name]["e2e"] = e["e2e"]
+            elif e["parity"] is not None:
+                others[name]["parity"] = e["parity"]
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
-
-    value = whole_job_value(rows, trials, args.steps, world, ms)
-    kernel_ms = ms_kernel / args.steps
-    if exact:
-        peak, peak_sus, peak_src = _peak_tensor()
-        flops = 2.0 * rows * cfg.n * cfg.N
-        achieved = flops / (kernel_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                    "traffic": None, "kernel_ms": kernel_ms, "flops_per_launch": flops, "peak_source": peak_src,
-                    "frac_of_sustained_peak": achieved / peak_sus,
-                    "kernels": "exact_operand_kernel + exact_tc_kernel (row sums in its epilogue)"}
-    else:
-        peak, peak_src = _peaks()
-        algo_bytes = rows * row_bytes
-        achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-        traffic = NCU_TRAFFIC["bytes_per_launch"] if (args.workload == WORKLOAD and
-                                                      NCU_TRAFFIC["sources_sha256"] == _kernel_sources_hash()) else None
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": traffic, "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": algo_bytes,
-                    "peak_source": peak_src,
-                    "kernels": "rdk_row_kernel (shared prior)" if args.prior else "rdk_stream_kernel + rdk_draw_kernel"}
-        if args.prior:
-            roofline["traffic"] = None
-
-    cpu = None
-    if not args.no_cpu_baseline and not exact and not args.prior:
-        cpu_value, cpu_dt, cpu_rows = _cpu_baseline(cfg)
-        cpu = {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"{cpu_rows} rows of {args.workload} through oracle.rdk_row (float64 numpy, one thread, {cpu_dt:.1f} s)"}
-
-    what = ("exact RDK on tensor cores (bf16 affinity, fp32 accumulate) + sampling/verification" if exact
-            else "linear RDK with one shared prior row in Eq. rdk-taylor + sampling/verification" if args.prior
-            else "linear RDK (first-order redistribution + sampling/verification)")
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {what}, N={cfg.N}, n={cfg.n}, batch={cfg.batch}, "
-                               f"positions={cfg.positions} (rows={rows}), bf16 inputs, trials={trials}",
-                   "rows_per_step": rows, "parallelism": f"replicas x{world} (no collective)",
-                   "l2": (f"operands of one step ({(cfg.N * cfg.n * 2 + rows * cfg.N * 4) / 1e6:.0f} MB) exceed the 126 MB L2"
-                          if exact else
-                          f"inputs rotate over {nsets} distinct batches ({nsets * rows * row_bytes / 1e6:.0f} MB > 126 MB L2)")},
-        "roofline": roofline,
-        "cpu_baseline": cpu,
-        "e2e": e2e,
-        "gpu_launches": launches_per_step * args.steps,
-        "clocks": sampler.summary(),
+        "config": head["config"], "timed": head["timed"], "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"],
+        "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "clocks": head["clocks"], "parity": head["parity"],
     }
-    if prep_ms is not None:
-        line["config"]["preprocessing_ms"] = prep_ms
+    if others:
+        line["workloads"] = others
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -398,12 +569,13 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["C2", "C3", "C4", "C5"], default=WORKLOAD,
-                    help="C2 (default) is the benchmark; C3/C4 are the other linear-path sizes, C5 the exact "
-                         "tensor-core path (used for profiling)")
+                    help="the headline workload of the line (default C2, the one the metric is quoted on); the others "
+                         "ride along under \"workloads\"")
+    ap.add_argument("--only", action="store_true", help="time the headline workload only (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     ap.add_argument("--prior", action="store_true",
                     help="linear workloads: time the variant with a shared static prior inside Eq. rdk-taylor "

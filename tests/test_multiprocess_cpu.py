@@ -61,3 +61,17 @@ def test_reference_arm_prints_on_rank_zero_only():
     line = json.loads(outs[0].splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["cpu_baseline"]["kind"] == "oracle"
+
+
+def test_timed_region_is_long_enough_whatever_the_step_count():
+    """The benchmark repeats its K-step loop until half a second has been timed and at least five times,
+    and reports the median; a handful of steps of a 50 microsecond kernel must not be the whole record."""
+    import bench
+    assert bench.repeats_for(0.05, 20) == 500          # 20 steps of 0.05 ms: 1 ms per loop
+    assert bench.repeats_for(0.05, 2000) == 5          # 100 ms per loop: the minimum of five
+    assert bench.repeats_for(0.4, 100) == 13
+    assert bench.repeats_for(1e-9, 1) == 2000          # capped
+    med, spread = bench.median_and_spread([1.0, 1.2, 0.9, 1.1, 1.0])
+    assert med == 1.0 and abs(spread - 0.3) < 1e-12
+    med, _ = bench.median_and_spread([2.0, 4.0])
+    assert med == 3.0
