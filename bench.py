@@ -29,7 +29,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 WORKLOAD = "C2"              # the configuration the metric is quoted on (--workload picks another as the headline)
-OTHER_WORKLOADS = ("C3", "C4", "C5")
+OTHER_WORKLOADS = ("C3", "C4", "C5", "T1")
 N_BUFFER_SETS = 6            # distinct input batches rotated through, so every step reads HBM
 METRIC = "verified draft tokens/sec"
 UNIT = "tokens/s"
@@ -506,6 +506,42 @@ def _parity_in_this_run(ctx: Ctx, cfg, s0, outs, index, kind, ws, nrows: int = 1
     return res
 
 
+def acceptance_report(ctx: Ctx, name: str = "T1"):
+    """Mean acceptance rate alpha = sum_j min(p_j, q~_j) of the three schemes of Sec. 5.2 ("Acceptance recovery") on
+    the heavy-tailed extreme-pruning workload, every alpha computed by the library's kernels on the same rows:
+    (a) pruning without redistribution: the unpruned drafter's q masked to the kept ids, not renormalised
+        (precomputed-w mode with RDK_FLAG_W_AS_GIVEN); (b) TLI: q' at the kept ids (precomputed-w mode);
+    (c) first-order RDK (the linear mode)."""
+    torch, B, W = ctx.torch, ctx.B, ctx.W
+    cfg = W.CONFIGS[name]
+    inp = W.make_inputs(cfg, device=str(ctx.dev), with_full_drafter=True)
+    kid = inp["kept_ids"].long()
+    index = B.rdk_prepare_ids(inp["kept_ids"], cfg.N)
+    rdk = B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, inp["target"], inp["drafter"], None, inp["uniforms"],
+                                  cfg.batch, cfg.positions)
+    w = torch.zeros(cfg.rows, cfg.N, dtype=torch.float32, device=ctx.dev)
+    w[:, kid] = torch.softmax(inp["drafter"].float(), dim=-1)
+    tli = B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, inp["target"], None, w, inp["uniforms"],
+                                  cfg.batch, cfg.positions)
+    q_full = torch.softmax(inp["drafter_full"].float(), dim=-1)
+    w.zero_()
+    w[:, kid] = q_full[:, kid]
+    prune = B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, inp["target"], None, w, inp["uniforms"],
+                                    cfg.batch, cfg.positions, flags=B.RDK_FLAG_W_AS_GIVEN)
+    torch.cuda.synchronize()
+    for o in (rdk, tli, prune):
+        B.check_status_word(o, f"acceptance report {name}")
+    p_kept = torch.softmax(inp["target"].float(), dim=-1)[:, kid].sum(-1)
+    mean = lambda t: float(t.double().mean())
+    return {"workload": f"{name}: N={cfg.N}, n={cfg.n}, rows={cfg.rows}, Student-t (5 d.o.f.) logit noise, Zipf bias, bf16",
+            "mean_alpha": {"pruning_without_redistribution": mean(prune["alpha"]), "tli": mean(tli["alpha"]),
+                           "taylor_rdk": mean(rdk["alpha"])},
+            "mean_drafter_mass_kept": mean(prune["S"]), "mean_target_mass_on_kept_ids": mean(p_kept),
+            "mean_theta": mean(rdk["theta"]),
+            "note": "alpha from the library's kernels (linear mode; precomputed-w mode for the two baselines); the first-order "
+                    "formula moves about theta / N of the drafter's mass off the kept ids, so (b) and (c) differ by about that"}
+
+
 def run_ours(args):
     import torch
 
@@ -547,6 +583,9 @@ def run_ours(args):
                 others[name]["e2e"] = e["e2e"]
             elif e["parity"] is not None:
                 others[name]["parity"] = e["parity"]
+    acceptance = None
+    if rank == 0 and not args.prior and (not args.only or args.workload == "T1"):
+        acceptance = acceptance_report(ctx)
 
     if rank != 0:
         if dist is not None:
@@ -561,6 +600,8 @@ def run_ours(args):
     }
     if others:
         line["workloads"] = others
+    if acceptance is not None:
+        line["acceptance"] = acceptance
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -572,7 +613,7 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["C2", "C3", "C4", "C5"], default=WORKLOAD,
+    ap.add_argument("--workload", choices=["C2", "C3", "C4", "C5", "T1"], default=WORKLOAD,
                     help="the headline workload of the line (default C2, the one the metric is quoted on); the others "
                          "ride along under \"workloads\"")
     ap.add_argument("--only", action="store_true", help="time the headline workload only (profiling runs)")

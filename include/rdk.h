@@ -66,6 +66,14 @@ typedef enum rdk_mode { RDK_MODE_LINEAR = 0, RDK_MODE_PRECOMPUTED_W = 1 } rdk_mo
  * kernel even where the streaming kernel would serve (the two can then be compared on the same
  * inputs; the row kernel divides exactly where the streaming kernel expands 1 / (N + p_j)).      */
 #define RDK_FLAG_ROW_KERNEL 1
+/* RDK_FLAG_W_AS_GIVEN (mode RDK_MODE_PRECOMPUTED_W only; RDK_ERR_INVALID_ARG elsewhere): q~ = w
+ * itself instead of w / sum(w).  For a w whose entries are probabilities of a larger distribution
+ * and sum to less than 1: the pruning-without-redistribution scheme of Sec. 5.2 ("Acceptance
+ * recovery", scheme (a)), where the drafter's full-vocabulary q is masked to I and not
+ * renormalised.  alpha, the rejection test and the residual max(0, p - w) then use w as it
+ * stands; the draft token is still drawn in proportion to w (a draw needs a distribution); the S
+ * output remains sum(w).  The caller guarantees 0 <= w_j and sum(w) <= 1.                         */
+#define RDK_FLAG_W_AS_GIVEN 2
 
 /* Which kernel a call of the linear mode takes (see rdk_sample_route).                           */
 typedef enum rdk_route { RDK_ROUTE_ROW_KERNEL = 0, RDK_ROUTE_STREAM_KERNEL = 1 } rdk_route;
@@ -85,7 +93,7 @@ typedef struct rdk_problem {
     int32_t target_dtype;       /* rdk_dtype of the target logits                                */
     int32_t drafter_dtype;      /* rdk_dtype of the drafter logits / probabilities               */
     int32_t drafter_kind;       /* rdk_kind: RDK_LOGITS are soft-maxed, RDK_PROBS taken as is    */
-    int32_t flags;              /* 0, or RDK_FLAG_ROW_KERNEL                                     */
+    int32_t flags;              /* 0, or an OR of RDK_FLAG_ROW_KERNEL, RDK_FLAG_W_AS_GIVEN       */
     int64_t target_row_stride;  /* elements between target rows; 0 means N                       */
     int64_t drafter_row_stride; /* elements between drafter rows; 0 means n                      */
     const void* kept_index;     /* device buffer filled by rdk_prepare_ids for this (N, n)       */
@@ -221,26 +229,28 @@ int rdk_redistribute_linear(const rdk_problem* problem, const void* target, cons
  *   trials     >= 1 independent draws per row (each uses its own 4 uniforms)
  *   out        see rdk_outputs
  *   ws         device workspace of rdk_sample_workspace_bytes(problem, mode, trials) bytes, 256-byte
- *              aligned (may be NULL when that size is 0).  The streaming kernel keeps there one
+ *              aligned (may be NULL when that size is 0).  The streaming kernels keep there one
  *              record of 4160 bytes per row (row scalars and per-segment sums of w, min(p, q~),
- *              max(0, p - q~), p), one 8-byte counter per (sequence, trial), and 64 bytes per
+ *              max(0, p - q~), p), one 4-byte counter per (sequence, trial), and 64 bytes per
  *              (row, CTA sharing the row) through which those CTAs exchange their partial
- *              soft-max sums and tell one another that a row's sums are written.  Its contents
- *              need no initialisation.  One workspace serves one call at a time: calls that
- *              share it must be ordered on one stream (they may be queued back to back without
- *              synchronising).  The call may be captured in a CUDA graph and the graph replayed:
- *              the kernel wipes the exchanged records of a row once the row is drawn, so a
- *              replay never meets the previous replay's.
+ *              soft-max sums.  Its contents need no initialisation.  One workspace serves one call
+ *              at a time: calls that share it must be ordered on one stream (they may be queued
+ *              back to back without synchronising).  The call may be captured in a CUDA graph and
+ *              the graph replayed: the second kernel wipes the exchanged records of a row once the
+ *              row is drawn, so a replay never meets the previous replay's.
  * Kernels.  For N >= 4096 with ascending valid kept ids, 16-byte aligned target rows, a 16-byte
- * aligned drafter base and an even drafter row stride, the linear mode is ONE persistent kernel
- * (launched cooperatively, one CTA per SM) that streams every row from HBM once; there the
- * quotient 1 / (N + p_j) is expanded in x = p_j / N <= 2^-12 and terms of relative size x^2
- * (below 2^-24) are dropped.  Every other problem takes the one-CTA-per-row kernel (three sweeps
- * over the row, exact division), which is several times slower; rdk_sample_route tells which
- * one a call would take and why.  The streaming kernel is launched with programmatic stream
- * serialisation: it may set itself up while the previous kernel of the stream drains, but reads
- * none of its inputs and touches nothing of the workspace before that kernel is complete, so
- * inputs written by the kernel queued just before the call are safe.
+ * aligned drafter base and an even drafter row stride, the linear mode is TWO launches: a
+ * persistent kernel (launched cooperatively, one CTA per SM) that streams every row from HBM once
+ * and leaves the per-row record above, and a small kernel (one CTA per row and trial) that draws
+ * the draft token, tests it and draws the replacement from those records, reading again only the
+ * few 1024-token chunks the draws fall into.  There the quotient 1 / (N + p_j) is expanded in
+ * x = p_j / N <= 2^-12 and terms of relative size x^2 (below 2^-24) are dropped.  Every other
+ * problem takes the one-CTA-per-row kernel (three sweeps over the row, exact division), which is
+ * several times slower; rdk_sample_route tells which one a call would take and why.  Both
+ * streaming kernels are launched with programmatic stream serialisation: each may set itself up
+ * while the previous kernel of the stream drains, but reads none of its inputs and touches nothing
+ * of the workspace before that kernel is complete, so inputs written by the kernel queued just
+ * before the call are safe.
  * If a bounded wait inside the kernel expires, out->status_word is set to RDK_ERR_TIMEOUT and the
  * outputs of that call are not valid.  Arithmetic of the linear mode: fp32.
  * ------------------------------------------------------------------------------------------- */
@@ -268,7 +278,7 @@ int rdk_sample_route(const rdk_problem* problem, int32_t mode, const void* targe
  * Every wait inside the streaming kernel (on a shared-memory barrier, on a record another CTA
  * publishes) gives up after a number of failed tries, records RDK_ERR_TIMEOUT in
  * out->status_word and lets the kernel run to its end.  This sets that number for later calls of
- * this process; 0 restores the default (2^20).  With a limit of 1 the waits of an ordinary call
+ * this process; 0 restores the default (2^17 tries of up to 2 us each).  With a limit of 1 the waits of an ordinary call
  * run out, which is how the tests reach the failure path without hanging or faulting anything.
  * ------------------------------------------------------------------------------------------- */
 void rdk_test_set_spin_limit(uint32_t limit);

@@ -25,6 +25,7 @@ RDK_LOGITS, RDK_PROBS = 0, 1
 RDK_MODE_LINEAR, RDK_MODE_PRECOMPUTED_W = 0, 1
 RDK_AFF_F32_ROWS, RDK_AFF_BF16_COLS = 0, 1
 RDK_FLAG_ROW_KERNEL = 1
+RDK_FLAG_W_AS_GIVEN = 2
 RDK_ROUTE_ROW_KERNEL, RDK_ROUTE_STREAM_KERNEL = 0, 1
 
 EXPORTS = [

@@ -154,7 +154,7 @@ extern "C" int rdk_redistribute_exact(const rdk_problem* problem, const void* dr
     }
     if (problem->N < 1 || problem->n < 1 || problem->batch < 1 || problem->positions < 1 || !problem->kept_index ||
         (problem->drafter_dtype != RDK_F32 && problem->drafter_dtype != RDK_BF16) ||
-        (problem->drafter_kind != RDK_LOGITS && problem->drafter_kind != RDK_PROBS) || (problem->flags & ~RDK_FLAG_ROW_KERNEL) != 0 ||
+        (problem->drafter_kind != RDK_LOGITS && problem->drafter_kind != RDK_PROBS) || (problem->flags & ~(RDK_FLAG_ROW_KERNEL | RDK_FLAG_W_AS_GIVEN)) != 0 ||
         (problem->drafter_row_stride != 0 && problem->drafter_row_stride < problem->n) || M->reserved != 0) {
         set_error("rdk_redistribute_exact: bad problem description");
         return RDK_ERR_INVALID_ARG;

@@ -236,7 +236,7 @@ rdk_row_kernel(const RowParams P) {
     __syncthreads();
     const double S_d = bc_d[0];
     const float S = (float)S_d;
-    c.inv_s = 1.f / S;
+    c.inv_s = (MODE == RDK_MODE_PRECOMPUTED_W && P.w_as_given) ? 1.f : 1.f / S;
 
     // ---- pass 3: alpha = sum min(p, q~), residual sums, optional q~ output ----------------------
     float* qrow = P.qtilde ? P.qtilde + (long long)row * P.N : nullptr;
@@ -417,7 +417,7 @@ static int validate_problem(const rdk_problem* pb, const char* who, bool need_in
     if ((long long)pb->batch * pb->positions > 0x7fffffffLL) { set_error("%s: too many rows", who); return RDK_ERR_INVALID_ARG; }
     if ((pb->target_dtype != RDK_F32 && pb->target_dtype != RDK_BF16) ||
         (pb->drafter_dtype != RDK_F32 && pb->drafter_dtype != RDK_BF16) ||
-        (pb->drafter_kind != RDK_LOGITS && pb->drafter_kind != RDK_PROBS) || (pb->flags & ~RDK_FLAG_ROW_KERNEL) != 0) {
+        (pb->drafter_kind != RDK_LOGITS && pb->drafter_kind != RDK_PROBS) || (pb->flags & ~(RDK_FLAG_ROW_KERNEL | RDK_FLAG_W_AS_GIVEN)) != 0) {
         set_error("%s: bad dtype / kind / flags field", who);
         return RDK_ERR_INVALID_ARG;
     }
@@ -442,6 +442,11 @@ static int run_rows(const rdk_problem* pb, int mode, const void* target, const v
     P.w = w; P.w_stride = w_stride ? w_stride : pb->N;
     P.uniforms = uniforms;
     P.prior = prior; P.prior_stride = prior_stride;
+    P.w_as_given = (pb->flags & RDK_FLAG_W_AS_GIVEN) ? 1 : 0;
+    if (P.w_as_given && mode != RDK_MODE_PRECOMPUTED_W) {
+        set_error("RDK_FLAG_W_AS_GIVEN applies to RDK_MODE_PRECOMPUTED_W only");
+        return RDK_ERR_INVALID_ARG;
+    }
     if (mode == RDK_MODE_LINEAR) {
         KeptIndexView v = make_view(pb->kept_index, pb->N, pb->n);
         P.header = v.header; P.mask = v.mask; P.rank = v.rank; P.slot = v.slot; P.ids = v.ids;
@@ -534,6 +539,10 @@ extern "C" int rdk_sample_route(const rdk_problem* problem, int32_t mode, const 
     int st = validate_problem(problem, "rdk_sample_route", mode == RDK_MODE_LINEAR);
     if (st != RDK_OK) return -st;
     if (mode != RDK_MODE_LINEAR) { if (why) *why = "precomputed w"; return RDK_ROUTE_ROW_KERNEL; }
+    if (problem->flags & RDK_FLAG_W_AS_GIVEN) {
+        set_error("RDK_FLAG_W_AS_GIVEN applies to RDK_MODE_PRECOMPUTED_W only");
+        return -RDK_ERR_INVALID_ARG;
+    }
     if (problem->flags & RDK_FLAG_ROW_KERNEL) { if (why) *why = "RDK_FLAG_ROW_KERNEL is set"; return RDK_ROUTE_ROW_KERNEL; }
     RowParams P{};
     P.N = problem->N; P.n = problem->n; P.rows = problem->batch * problem->positions; P.trials = trials;

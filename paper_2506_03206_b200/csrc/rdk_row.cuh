@@ -19,6 +19,7 @@ struct RowParams {
     float* alpha; float* theta; float* S; float* residual_mass; float* qtilde;
     int32_t* status_word;
     int num_tiles;
+    int w_as_given;        // precomputed-w mode: q~ = w itself (no division by its sum)
     // streaming path only
     int positions;
     int32_t* accepted_len;

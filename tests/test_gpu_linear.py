@@ -438,16 +438,93 @@ def test_full_size_configs_sampled_rows(name, nrows):
     assert abs(acc.double().mean().item() - mean_alpha) < 5 * sigma + 1e-3
 
 
-def test_extreme_pruning_heavy_tailed_logits_and_tli_baseline():
-    """200k vocabulary, 500 kept tokens, Student-t logits (the shape of the paper's synthetic
-    experiment): parity of the linear path on sampled rows, and the TLI baseline (q~ = q', obtained by
-    handing the sampler w = q' scattered to the full vocabulary) next to it."""
+def _masked_drafter(inp, cfg):
+    """Scheme (a) of Sec. 5.2: the unpruned drafter's soft-max, zero outside the kept ids, not renormalised."""
+    q_full = torch.softmax(inp["drafter_full"].float(), dim=-1)
+    w = torch.zeros(cfg.rows, cfg.N, dtype=torch.float32, device=q_full.device)
+    kid = inp["kept_ids"].long()
+    w[:, kid] = q_full[:, kid]
+    return w
+
+
+def _check_w_as_given(rdk, cfg, inp, w, out, rows):
+    """RDK_FLAG_W_AS_GIVEN against the checker's primitives with q~ = w, un-normalised: alpha (Definition 2.1), the
+    draw in proportion to w, the rejection test and the residual (Algorithm 4 steps 4-8)."""
+    t = PU.Tally()
+    for r in rows:
+        p = O.softmax(W.to_f64(inp["target"][r]))
+        wr = W.to_f64(w[r])
+        u = inp["uniforms"][r].cpu().numpy().astype(np.float64)
+        assert abs(float(out["alpha"][r]) - O.acceptance_rate(p, wr)) < PU.ABS_TOL
+        R, _ = O.residual(p, wr)
+        assert abs(float(out["residual_mass"][r]) - R) < PU.ABS_TOL
+        assert abs(float(out["S"][r]) - wr.sum()) < PU.ABS_TOL
+        for k in range(cfg.trials):
+            d = O.inverse_cdf(wr, u[k, 0])
+            got_d = int(out["draft_token"][r * cfg.trials + k])
+            if got_d != d:
+                cdf = np.cumsum(wr)
+                thr = u[k, 0] * cdf[-1]
+                lo = cdf[got_d - 1] if got_d > 0 else 0.0
+                assert min(abs(thr - lo), abs(thr - cdf[got_d])) <= PU.ABS_TOL * cdf[-1], (r, k, d, got_d)
+                t.ambiguous_draft += 1
+                continue
+            a, acc = O.accept_test(p, wr, d, u[k, 1])
+            assert abs(float(out["accept_prob"][r * cfg.trials + k]) - a) < 1e-4
+            if bool(out["accepted"][r * cfg.trials + k]) != acc:
+                assert abs(u[k, 1] * wr[d] - p[d]) <= PU.ABS_TOL * max(p[d], wr[d])
+                t.ambiguous_accept += 1
+                continue
+            want = d if acc else O.residual_sample(p, wr, u[k, 2])
+            got = int(out["out_token"][r * cfg.trials + k])
+            if got != want:
+                cr = np.cumsum(np.maximum(0.0, p - wr))
+                thr = u[k, 2] * cr[-1]
+                lo = cr[got - 1] if got > 0 else 0.0
+                assert min(abs(thr - lo), abs(thr - cr[got])) <= PU.ABS_TOL * cr[-1], (r, k, want, got)
+                t.ambiguous_residual += 1
+        t.draws += cfg.trials
+    return t
+
+
+def test_pruning_without_redistribution_keeps_w_as_given():
+    """Scheme (a) of Sec. 5.2 on a small problem, several trials per row: with RDK_FLAG_W_AS_GIVEN the sampler
+    verifies against the masked, un-normalised drafter distribution; the flag is refused in the linear mode."""
+    rdk = _rdk()
+    B = rdk.binding
+    cfg = W.tiny_config(N=5003, n=311, rows=7, dtype="bf16", trials=8, rho=0.8, seed=77)
+    inp = W.make_inputs(cfg, device="cuda", with_full_drafter=True)
+    idx = rdk.rdk_prepare_ids(inp["kept_ids"], cfg.N)
+    w = _masked_drafter(inp, cfg)
+    assert torch.all(w.sum(-1) < 0.999)                 # mass was pruned away: this is not TLI
+    out = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_PRECOMPUTED_W, inp["target"], None, w, inp["uniforms"],
+                                    cfg.batch, cfg.positions, flags=B.RDK_FLAG_W_AS_GIVEN)
+    torch.cuda.synchronize()
+    t = _check_w_as_given(rdk, cfg, inp, w, out, range(cfg.rows))
+    t.assert_ok()
+    # without the flag the same w is renormalised (TLI of the masked drafter): a different alpha
+    out_n = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_PRECOMPUTED_W, inp["target"], None, w, inp["uniforms"],
+                                      cfg.batch, cfg.positions)
+    torch.cuda.synchronize()
+    assert torch.all(out_n["alpha"] > out["alpha"] + 1e-4)
+    with pytest.raises(Exception, match="W_AS_GIVEN"):
+        rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, inp["target"], inp["drafter"], None, inp["uniforms"],
+                                  cfg.batch, cfg.positions, flags=B.RDK_FLAG_W_AS_GIVEN)
+
+
+def test_extreme_pruning_heavy_tailed_logits_three_schemes():
+    """200k vocabulary, 500 kept tokens, Student-t logits (the shape of the synthetic experiment of Sec. 5.2):
+    parity of the linear path on every row, and the two baselines next to it through the precomputed-w mode:
+    TLI (w = q' scattered to the full vocabulary) and pruning without redistribution (w = the unpruned
+    drafter's q masked to the kept ids, RDK_FLAG_W_AS_GIVEN)."""
     rdk = _rdk()
     B = rdk.binding
     cfg = W.CONFIGS["T1"]
-    inp = W.make_inputs(cfg, device="cuda")
+    inp = W.make_inputs(cfg, device="cuda", with_full_drafter=True)
     rows = list(range(cfg.rows))
-    _run_linear(cfg, inp, rows=rows, check_qtilde=False).assert_ok_at_scale(cfg.n)
+    t = _run_linear(cfg, inp, rows=rows, check_qtilde=False)
+    t.assert_ok_at_scale(cfg.n)
+    t.record("T1 linear, all rows")
     idx = rdk.rdk_prepare_ids(inp["kept_ids"], cfg.N)
     out_rdk = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_LINEAR, inp["target"], inp["drafter"], None, inp["uniforms"],
                                         cfg.batch, cfg.positions)
@@ -457,15 +534,21 @@ def test_extreme_pruning_heavy_tailed_logits_and_tli_baseline():
     w[:, inp["kept_ids"].long()] = qp
     out_tli = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_PRECOMPUTED_W, inp["target"], None, w, inp["uniforms"],
                                         cfg.batch, cfg.positions)
+    wm = _masked_drafter(inp, cfg)
+    out_prune = rdk.rdk_sample_and_verify(idx, B.RDK_MODE_PRECOMPUTED_W, inp["target"], None, wm, inp["uniforms"],
+                                          cfg.batch, cfg.positions, flags=B.RDK_FLAG_W_AS_GIVEN)
     torch.cuda.synchronize()
     kappa = inp["kept_ids"].cpu().numpy()
     for r in rows[::8]:
         p = O.softmax(W.to_f64(inp["target"][r]))
         q_tli = O.tli_project(W.to_f64(w[r])[kappa], kappa, cfg.N)
         assert abs(float(out_tli["alpha"][r]) - O.acceptance_rate(p, q_tli)) < PU.ABS_TOL
-    a_rdk, a_tli = out_rdk["alpha"].double(), out_tli["alpha"].double()
+    _check_w_as_given(rdk, cfg, inp, wm, out_prune, rows[::8])
+    a_rdk, a_tli, a_prune = out_rdk["alpha"].double(), out_tli["alpha"].double(), out_prune["alpha"].double()
     # the first-order formula moves only about theta / N of the mass: both rates agree to ~1e-5 here
     assert torch.all((a_rdk - a_tli).abs() < 1e-4)
+    # masking shrinks every kept probability, renormalising can only raise min(p, q) term by term
+    assert torch.all(a_prune <= a_tli + 1e-6)
 
 
 @pytest.mark.parametrize("dtype,N,n,kind", [("bf16", 5000, 900, "logits"), ("f32", 1001, 77, "logits"),

@@ -107,7 +107,10 @@ def test_route_query_reports_host_side_argument_errors(B):
     pb.flags = B.RDK_FLAG_ROW_KERNEL
     assert L.rdk_sample_route(C.byref(pb), 0, None, None, 1, None, 0, C.byref(why)) == B.RDK_ROUTE_ROW_KERNEL
     assert b"RDK_FLAG_ROW_KERNEL" in why.value
-    pb.flags = 2
+    pb.flags = B.RDK_FLAG_W_AS_GIVEN          # belongs to the precomputed-w mode only
+    assert L.rdk_sample_route(C.byref(pb), 0, None, None, 1, None, 0, None) == -B.RDK_ERR_INVALID_ARG
+    assert L.rdk_sample_route(C.byref(pb), 1, None, None, 1, None, 0, None) == B.RDK_ROUTE_ROW_KERNEL
+    pb.flags = 4                              # not a flag
     assert L.rdk_sample_route(C.byref(pb), 0, None, None, 1, None, 0, None) == -B.RDK_ERR_INVALID_ARG
     # an index this process never prepared at that address: not known to be ascending
     pb.flags = 0

@@ -129,7 +129,8 @@ def embeddings(cfg: RDKConfig, device: str = "cpu") -> torch.Tensor:
 
 
 def make_inputs(cfg: RDKConfig, device: str = "cpu", variant: int = 0,
-                with_embeddings: bool = False, row_chunk: int = 128) -> Dict[str, object]:
+                with_embeddings: bool = False, row_chunk: int = 128,
+                with_full_drafter: bool = False) -> Dict[str, object]:
     """Draw one batch of inputs for ``cfg``.
 
     Returns a dict with
@@ -138,6 +139,8 @@ def make_inputs(cfg: RDKConfig, device: str = "cpu", variant: int = 0,
       drafter   dtype [rows, n]               drafter logits y (or probabilities, C5)
       uniforms  float32 [rows, trials, 4]     Philox uniforms
       embeddings dtype [N, emb_dim]           only when with_embeddings
+      drafter_full dtype [rows, N]            only when with_full_drafter (logit workloads): the logits of
+                                              the drafter before pruning, equal to ``drafter`` at the kept ids
     ``variant`` selects an independent batch of the same workload (used to rotate buffers).
     """
     dev = torch.device(device)
@@ -154,12 +157,19 @@ def make_inputs(cfg: RDKConfig, device: str = "cpu", variant: int = 0,
     target = torch.empty(rows, N, dtype=dt, device=dev)
     drafter = torch.empty(rows, n, dtype=dt, device=dev)
     c = math.sqrt(max(0.0, 1.0 - cfg.rho * cfg.rho))
-    def noise(*shape):
-        x = torch.randn(*shape, generator=g, device=dev, dtype=torch.float32)
+    if with_full_drafter and cfg.drafter_kind == "probs":
+        raise ValueError("with_full_drafter is defined for the logit workloads only")
+    # the pruned-away part of the drafter comes from a generator of its own, so that asking for it
+    # leaves every other tensor of the batch as it was
+    g_full = _gen(cfg.seed * 7919 + 13 + 1000003 * variant, dev) if with_full_drafter else None
+    drafter_full = torch.empty(rows, N, dtype=dt, device=dev) if with_full_drafter else None
+    def noise(*shape, gen=None):
+        gen = g if gen is None else gen
+        x = torch.randn(*shape, generator=gen, device=dev, dtype=torch.float32)
         if cfg.noise == "student_t5":     # t_5 = normal / sqrt(chi2_5 / 5), rescaled to unit variance (var of t_5 is 5/3)
             chi2 = torch.zeros(*shape, device=dev, dtype=torch.float32)
             for _ in range(5):
-                chi2 += torch.randn(*shape, generator=g, device=dev, dtype=torch.float32) ** 2
+                chi2 += torch.randn(*shape, generator=gen, device=dev, dtype=torch.float32) ** 2
             x = x / torch.sqrt(chi2 / 5.0) * math.sqrt(3.0 / 5.0)
         return x
 
@@ -180,11 +190,17 @@ def make_inputs(cfg: RDKConfig, device: str = "cpu", variant: int = 0,
             y = bias[kidl] + cfg.sigma * (cfg.rho * gz[:, kidl] + c * h)
             target[r0:r1] = z.to(dt)
             drafter[r0:r1] = y.to(dt)
+            if with_full_drafter:
+                yf = bias + cfg.sigma * (cfg.rho * gz + c * noise(r1 - r0, N, gen=g_full))
+                yf[:, kidl] = y
+                drafter_full[r0:r1] = yf.to(dt)
     u = torch.from_numpy(philox_uniforms(cfg.seed + 104729 * variant, rows, cfg.trials)).to(dev)
     out: Dict[str, object] = {"cfg": cfg, "kept_ids": kid, "target": target, "drafter": drafter,
                               "uniforms": u}
     if with_embeddings:
         out["embeddings"] = embeddings(cfg, device)
+    if with_full_drafter:
+        out["drafter_full"] = drafter_full
     return out
 
 
