@@ -16,15 +16,15 @@ Notation (the paper reuses symbols; one name per object here):
   M      row-stochastic token-affinity matrix, n x N      (Eq. symbolic-m, rows i in I)
   w      un-normalised redistributed weights (the paper's p-tilde), S = sum_j w_j
   q~     redistributed drafter distribution w / S          (the paper's p', p_RDK, p_Taylor)
-  theta  p^T q'                                            (Sec. 4, "Let theta = p^T q'")
+  theta  p^T q'                                            (Sec. 4, defined just before Eq. rdk-taylor)
   alpha  acceptance rate sum_x min(p(x), q~(x))            (Definition 2.1)
 
 Conventions the paper leaves open and this checker fixes (each is a documented reading):
   * "Sample" (Algorithm 4) is inverse-CDF in ascending token id: the smallest j whose inclusive
     prefix sum C_j is strictly greater than u * C_last, u in [0, 1).  A zero-weight token can
     never be drawn.  If rounding leaves no such j, the last positive-weight token is taken.
-  * The rejection test of Algorithm 4 ("if p <= q reject with probability 1 - p/q") is taken as:
-    accepted  <=>  u2 * q~(d) < p(d).
+  * The rejection test of Algorithm 4 (a draft with p below q~ is turned down with the
+    complementary probability of p / q~) is taken as:  accepted  <=>  u2 * q~(d) < p(d).
   * The residual normaliser 1 - sum min(p, q~) is computed as the direct sum of max(0, p - q~);
     if that sum is not positive the replacement token is drawn from p.
   * kept ids < 0 or >= N stand for drafter tokens outside the target vocabulary (the set F of
@@ -188,7 +188,7 @@ def redistribute_linear(p: np.ndarray, qprime: np.ndarray):
 
 
 # ----------------------------------------------------------------------------------------------
-# O4  normalisation  (Eq. rdk-taylor, second part;  Algorithm 1 step 2 "such that sum p' = 1")
+# O4  normalisation  (Eq. rdk-taylor, second part;  Algorithm 1 step 2: the weights are scaled to sum to 1)
 # ----------------------------------------------------------------------------------------------
 def normalise(w: np.ndarray):
     """S = sum_j w_j (ascending j), q~ = w / S.  Returns (S, q~)."""
