@@ -240,7 +240,8 @@ int rdk_redistribute_linear(const rdk_problem* problem, const void* target, cons
  *              row is drawn, so a replay never meets the previous replay's.
  * Kernels.  For N >= 4096 with ascending valid kept ids, 16-byte aligned target rows, a 16-byte
  * aligned drafter base and an even drafter row stride, the linear mode is TWO launches: a
- * persistent kernel (launched cooperatively, one CTA per SM) that streams every row from HBM once
+ * persistent kernel (one CTA per SM; the first launch of a shape is a cooperative one, which proves
+ * that the grid fits the SMs at hand) that streams every row from HBM once
  * and leaves the per-row record above, and a small kernel (one CTA per row and trial) that draws
  * the draft token, tests it and draws the replacement from those records, reading again only the
  * few 1024-token chunks the draws fall into.  There the quotient 1 / (N + p_j) is expanded in

@@ -428,10 +428,85 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         for (int k = 0; k < 16; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&pbar[k])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // The load warp sets up the ring's barriers itself and starts the copies of the first rows' target slices
-    // right away (they need nothing from the index), so that HBM's first answer travels while the rest of the
-    // CTA is still setting up.  Only their byte count is announced here; the arrival that completes a stage's
-    // phase follows in the row loop, with the drafter copies.
+    // per-warp quantities of the streaming warps (taken from lane 0 so that the compiler knows they are uniform)
+    const int w_r0 = __shfl_sync(0xffffffffu, sd.x, 0), w_kcp = __shfl_sync(0xffffffffu, sd.y, 0);
+    const int w_gstart = __shfl_sync(0xffffffffu, sd.z, 0), w_dummy = __shfl_sync(0xffffffffu, sd.w, 0);
+    const int w_kcs = min(w_kcp, g.ycap);
+    const uint32_t pad2 = zslice | (zslice << 16);      // both slots at the spare -inf
+
+    // offsets (from the start of the slice, 16 bits each) of the target logits of this lane's two slots of every step:
+    // requested first of all, they travel while the rest of the set-up runs
+    uint32_t gor[NST > 0 ? NST : 1];
+    if (warp < kSW && NST > 0) {
+        const uint32_t* gt = reinterpret_cast<const uint32_t*>(g.goff + w_gstart);
+        const int npairs = ((w_kcp + 63) & ~63) >> 1;       // pairs tabulated for this segment
+#pragma unroll
+        for (int st = 0; st < (NST > 0 ? NST : 1); ++st) {
+            const int q = st * 32 + lane;
+            uint32_t o = q < npairs ? __ldg(gt + q) : pad2;
+            if (2 * q >= w_kcs) o = (o & 0xffff0000u) | zslice;            // beyond the cache: uncached route
+            if (2 * q + 1 >= w_kcs) o = (o & 0x0000ffffu) | (zslice << 16);
+            gor[st] = o;
+        }
+    } else {
+        gor[0] = 0u;
+    }
+
+    // ---- state of the load warp's ring (used by its prologue here and by its loop below) ----------------------
+    const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
+    const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
+    const int lenc_v = lenc & ~(kZPer - 1);
+    const uint32_t zbytes = (uint32_t)lenc_v * (uint32_t)sizeof(TZ);
+    const uint32_t kbytes = lane < kSW ? (uint32_t)min(sd.y, g.ycap) * (uint32_t)sizeof(TY) : 0u;
+    const uintptr_t y_end16 = reinterpret_cast<uintptr_t>(static_cast<const TY*>(P.drafter) +
+                                                          (long long)(P.rows - 1) * P.drafter_stride + P.n) & ~uintptr_t(15);
+    const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0c;
+    const TY* ny = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + sd.x;
+    const uint32_t l_yw_off = zslice + 16u + (uint32_t)(lane & (kSW - 1)) * (uint32_t)g.ystage;
+    int l_s = 0;
+    uint32_t l_eph = 1, l_st_a = dsm_a, l_fb = full_a, l_eb = empty_a;    // a fresh stage counts as released
+    unsigned char* l_st_p = dsm;
+    // one row: one bulk copy of the CTA's slice of the target row and one per warp of the matching drafter values,
+    // into the stage the streaming warps have released
+    auto load_row = [&]() {
+        mbar_wait(l_eb, l_eph, &fail, spin_limit);
+        // the few elements a 16-byte copy cannot cover go by plain stores: a slice that ends inside a
+        // vector, and the very end of the drafter buffer
+        const uintptr_t b0 = reinterpret_cast<uintptr_t>(ny), b1 = b0 + kbytes;
+        const uintptr_t a0 = b0 & ~uintptr_t(15);
+        uintptr_t a1 = (b1 + 15) & ~uintptr_t(15);
+        if (a1 > y_end16) a1 = y_end16 > a0 ? y_end16 : a0;     // never read past the drafter buffer
+        const uint32_t ybytes = kbytes ? (uint32_t)(a1 - a0) : 0u;
+        if (lane < lenc - lenc_v) reinterpret_cast<TZ*>(l_st_p)[lenc_v + lane] = nz[lenc_v + lane];
+        if (kbytes && a1 < b1) {
+            const uintptr_t t0 = a1 > b0 ? a1 : b0;
+            const int nt = (int)((b1 - t0) / sizeof(TY));
+            for (int k = 0; k < nt; ++k) reinterpret_cast<TY*>(l_st_p + l_yw_off + (t0 - a0))[k] = reinterpret_cast<const TY*>(t0)[k];
+        }
+        const uint32_t total = zbytes + __reduce_add_sync(0xffffffffu, ybytes);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage was last touched by plain loads and stores
+        if (lane == 0) {
+            if (total == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(l_fb) : "memory");
+            else asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(l_fb), "r"(total) : "memory");
+            for (uint32_t off = 0; off < zbytes; off += 32768u) {
+                const uint32_t sz = min(32768u, zbytes - off);
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(l_st_a + off), "l"(reinterpret_cast<const char*>(nz) + off), "r"(sz), "r"(l_fb) : "memory");
+            }
+        }
+        __syncwarp();
+        if (ybytes)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(l_st_a + l_yw_off), "l"(a0), "r"(ybytes), "r"(l_fb) : "memory");
+        nz += (long long)g.G * P.target_stride; ny += (long long)g.G * P.drafter_stride;
+        l_st_a += stage; l_st_p += stage; l_fb += 8u; l_eb += 8u;
+        if (++l_s == g.NS) { l_s = 0; l_eph ^= 1u; l_st_a = dsm_a; l_st_p = dsm; l_fb = full_a; l_eb = empty_a; }
+    };
+    // The load warp sets up the ring by itself and starts the first rows' copies right away, so that HBM's first
+    // answer travels while the rest of the CTA is still setting up: it initialises the ring's barriers, gives the
+    // parts of the stages that no copy writes their neutral values (beyond the vocabulary and the 16 spare bytes of
+    // every stage: weight 0; the drafter regions start out as weight 0 too -- slots beyond a copy keep whatever an
+    // earlier row left there, and are masked), and issues the first NS rows.
     const int pre_rows = min(g.NS, rows_g);
     if (warp == kWLoad) {
         if (lane == 0) {
@@ -441,69 +516,32 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             }
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
+        {
+            const uint32_t fill16 = KIND == RDK_LOGITS ? (sizeof(TY) == 2 ? 0xff80ff80u : 0xff800000u) : 0u;      // -inf, or 0
+            const uint32_t ninf16 = sizeof(TZ) == 2 ? 0xff80ff80u : 0xff800000u;
+            const uint32_t z0 = zbytes, z1 = zslice + 16u;        // [end of the copied vectors, spare bytes included)
+            for (int k = 0; k < g.NS; ++k) {
+                const uint32_t base = dsm_a + (uint32_t)k * stage;
+                for (uint32_t o = z0 + 16u * lane; o < z1; o += 512u)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + o), "r"(ninf16) : "memory");
+                for (uint32_t o = z1 + 16u * lane; o < stage; o += 512u)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + o), "r"(fill16) : "memory");
+            }
+        }
         __syncwarp();
         asm volatile("griddepcontrol.wait;" ::: "memory");     // the inputs may be the previous kernel's outputs
-        if (lane == 0) {
-            const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
-            const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
-            const uint32_t zbytes = (uint32_t)(lenc & ~(kZPer - 1)) * (uint32_t)sizeof(TZ);
-            const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0c;
-            for (int k = 0; k < pre_rows && zbytes; ++k) {
-                const uint32_t fb = full_a + 8u * (uint32_t)k, st_a = dsm_a + (uint32_t)k * stage;
-                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(fb), "r"(zbytes) : "memory");
-                for (uint32_t off = 0; off < zbytes; off += 32768u) {
-                    const uint32_t sz = min(32768u, zbytes - off);
-                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                 ::"r"(st_a + off), "l"(reinterpret_cast<const char*>(nz) + off), "r"(sz), "r"(fb) : "memory");
-                }
-                nz += (long long)g.G * P.target_stride;
-            }
-        }
-    }
-    // beyond the vocabulary, and the 16 spare bytes of every stage: weight 0; the drafter regions start
-    // out as weight 0 too (slots beyond a copy keep whatever an earlier row left there, and are masked)
-    {
-        const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
-        const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
-        const TY yfill = KIND == RDK_LOGITS ? neg_inf<TY>() : zero_of<TY>();
-        const int ycount = kSW * g.ystage / (int)sizeof(TY);
-        for (int k = 0; k < g.NS; ++k) {
-            TZ* zs = reinterpret_cast<TZ*>(dsm + (size_t)k * stage);
-            for (int t = lenc + tid; t < kSW * g.Lw + kZPer; t += kSThreads) zs[t] = neg_inf<TZ>();
-            TY* ysr = reinterpret_cast<TY*>(dsm + (size_t)k * stage + zslice + 16u);
-            for (int t = tid; t < ycount; t += kSThreads) ysr[t] = yfill;
-        }
+        for (int k = 0; k < pre_rows; ++k) load_row();
     }
 
-    // per-warp quantities of the streaming warps (taken from lane 0 so that the compiler knows they are uniform)
-    const int w_r0 = __shfl_sync(0xffffffffu, sd.x, 0), w_kcp = __shfl_sync(0xffffffffu, sd.y, 0);
-    const int w_gstart = __shfl_sync(0xffffffffu, sd.z, 0), w_dummy = __shfl_sync(0xffffffffu, sd.w, 0);
-    const int w_kcs = min(w_kcp, g.ycap);
-    const uint32_t pad2 = zslice | (zslice << 16);      // both slots at the spare -inf
-
-    // offsets (from the start of the slice, 16 bits each) of the target logits of this lane's two slots of every step
-    uint32_t gor[NST > 0 ? NST : 1];
-    if (warp < kSW) {
+    if (NST == 0 && warp < kSW) {          // the route with runtime loops keeps the offsets in shared memory
         const uint32_t* gt = reinterpret_cast<const uint32_t*>(g.goff + w_gstart);
-        const int npairs = ((w_kcp + 63) & ~63) >> 1;       // pairs tabulated for this segment
-        if (NST > 0) {
-#pragma unroll
-            for (int st = 0; st < (NST > 0 ? NST : 1); ++st) {
-                const int q = st * 32 + lane;
-                uint32_t o = q < npairs ? __ldg(gt + q) : pad2;
-                if (2 * q >= w_kcs) o = (o & 0xffff0000u) | zslice;            // beyond the cache: uncached route
-                if (2 * q + 1 >= w_kcs) o = (o & 0x0000ffffu) | (zslice << 16);
-                gor[st] = o;
-            }
-        } else {
-            const uint32_t gbase = dsm_a + off_goff + (uint32_t)warp * (uint32_t)g.ycap * 2u;
-            for (int q = lane; q < nst * 32; q += 32) {
-                uint32_t o = q < npairs ? __ldg(gt + q) : pad2;
-                if (2 * q >= w_kcs) o = (o & 0xffff0000u) | zslice;
-                if (2 * q + 1 >= w_kcs) o = (o & 0x0000ffffu) | (zslice << 16);
-                sts32(gbase + (uint32_t)q * 4u, o);
-            }
-            gor[0] = 0u;
+        const int npairs = ((w_kcp + 63) & ~63) >> 1;
+        const uint32_t gbase = dsm_a + off_goff + (uint32_t)warp * (uint32_t)g.ycap * 2u;
+        for (int q = lane; q < nst * 32; q += 32) {
+            uint32_t o = q < npairs ? __ldg(gt + q) : pad2;
+            if (2 * q >= w_kcs) o = (o & 0xffff0000u) | zslice;
+            if (2 * q + 1 >= w_kcs) o = (o & 0x0000ffffu) | (zslice << 16);
+            sts32(gbase + (uint32_t)q * 4u, o);
         }
     }
 
@@ -829,58 +867,8 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         }
     } else {
         // ================================ load warp =====================================================
-        // per row: one bulk copy of the CTA's slice of the target row and one per warp of the matching
-        // drafter values, into the stage the streaming warps have released
-        const int j0c = (int)min((long long)crank * kSW * g.Lw, (long long)P.N);
-        const int lenc = max(0, min(P.N - j0c, kSW * g.Lw));
-        const int lenc_v = lenc & ~(kZPer - 1);
-        const uint32_t zbytes = (uint32_t)lenc_v * (uint32_t)sizeof(TZ);
-        const int l_kcs = min(sd.y, g.ycap);
-        const uint32_t kbytes = lane < kSW ? (uint32_t)l_kcs * (uint32_t)sizeof(TY) : 0u;
-        const uintptr_t y_end16 = reinterpret_cast<uintptr_t>(static_cast<const TY*>(P.drafter) +
-                                                              (long long)(P.rows - 1) * P.drafter_stride + P.n) & ~uintptr_t(15);
-        const long long zstep = (long long)g.G * P.target_stride, ystep = (long long)g.G * P.drafter_stride;
-        const TZ* nz = static_cast<const TZ*>(P.target) + (long long)grp * P.target_stride + j0c;
-        const TY* ny = static_cast<const TY*>(P.drafter) + (long long)grp * P.drafter_stride + sd.x;
-        const uint32_t yw_off = zslice + 16u + (uint32_t)(lane & (kSW - 1)) * (uint32_t)g.ystage;
-        int s = 0;
-        uint32_t eph = 1, st_a = dsm_a, fb = full_a, eb = empty_a;    // a fresh stage counts as released
-        unsigned char* st_p = dsm;
-        for (int it = 0; it < rows_g; ++it) {
-            mbar_wait(eb, eph, &fail, spin_limit);
-            const bool z_issued = it < pre_rows;          // the target slice of this row is on its way already
-            // the few elements a 16-byte copy cannot cover go by plain stores: a slice that ends inside a
-            // vector, and the very end of the drafter buffer
-            const uintptr_t b0 = reinterpret_cast<uintptr_t>(ny), b1 = b0 + kbytes;
-            const uintptr_t a0 = b0 & ~uintptr_t(15);
-            uintptr_t a1 = (b1 + 15) & ~uintptr_t(15);
-            if (a1 > y_end16) a1 = y_end16 > a0 ? y_end16 : a0;     // never read past the drafter buffer
-            const uint32_t ybytes = kbytes ? (uint32_t)(a1 - a0) : 0u;
-            if (lane < lenc - lenc_v) reinterpret_cast<TZ*>(st_p)[lenc_v + lane] = nz[lenc_v + lane];
-            if (kbytes && a1 < b1) {
-                const uintptr_t t0 = a1 > b0 ? a1 : b0;
-                const int nt = (int)((b1 - t0) / sizeof(TY));
-                for (int k = 0; k < nt; ++k) reinterpret_cast<TY*>(st_p + yw_off + (t0 - a0))[k] = reinterpret_cast<const TY*>(t0)[k];
-            }
-            const uint32_t total = (z_issued ? 0u : zbytes) + __reduce_add_sync(0xffffffffu, ybytes);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage was last touched by plain loads and stores
-            if (lane == 0) {
-                if (total == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(fb) : "memory");
-                else asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(total) : "memory");
-                for (uint32_t off = 0; !z_issued && off < zbytes; off += 32768u) {
-                    const uint32_t sz = min(32768u, zbytes - off);
-                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                 ::"r"(st_a + off), "l"(reinterpret_cast<const char*>(nz) + off), "r"(sz), "r"(fb) : "memory");
-                }
-            }
-            __syncwarp();
-            if (ybytes)
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(st_a + yw_off), "l"(a0), "r"(ybytes), "r"(fb) : "memory");
-            nz += zstep; ny += ystep;
-            st_a += stage; st_p += stage; fb += 8u; eb += 8u;
-            if (++s == g.NS) { s = 0; eph ^= 1u; st_a = dsm_a; st_p = dsm; fb = full_a; eb = empty_a; }
-        }
+        // the first rows went out during the set-up; one row per stage as the streaming warps release them
+        for (int it = pre_rows; it < rows_g; ++it) load_row();
         if (ld_volatile_s32(&fail)) {
             // A wait gave up somewhere, so nobody may have waited for the last copies: let them land before
             // the CTA leaves (bounded as well, on a count of its own).
@@ -1145,21 +1133,35 @@ static cudaError_t launch_stream(const RowParams& P, StreamGeo g, cudaStream_t s
     cfg.blockDim = dim3(kSThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
+    // The CTAs of a group wait for one another, so all of the grid must be resident together.  A cooperative launch
+    // makes the driver guarantee that, at a price of about 4 us per launch.  It is asked for on the first launch of a
+    // (kernel, device, shared-memory size) only: that launch proves that the grid fits the SMs this context may
+    // use; later launches of the same shape are ordinary ones (one CTA per SM, grid <= the SM count), and should
+    // something else keep CTAs from becoming resident, their peers' bounded waits end in RDK_ERR_TIMEOUT.
+    static thread_local int v_dev = -1;
+    static thread_local size_t v_smem = 0;
+    const bool fits_proven = v_dev == dev && v_smem == smem;
     cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeCooperative;      // the CTAs of a group wait for one another: all must be resident
-    attr[0].val.cooperative = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set itself up while the previous kernel drains
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set itself up while the previous kernel drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
     static std::atomic<int> c_pdl{1};                 // whether the two attributes are accepted together on this system
     const int with_pdl = c_pdl.load();
-    cfg.numAttrs = with_pdl ? 2 : 1;
-    e = cudaLaunchKernelEx(&cfg, kern, P, g);
-    if (with_pdl && (e == cudaErrorNotSupported || e == cudaErrorInvalidValue)) {
-        (void)cudaGetLastError();
+    if (fits_proven) {
         cfg.numAttrs = 1;
         e = cudaLaunchKernelEx(&cfg, kern, P, g);
-        if (e == cudaSuccess) c_pdl.store(0);         // the pair is what this system refuses
+    } else {
+        if (!with_pdl) { attr[0] = attr[1]; cfg.numAttrs = 1; } else cfg.numAttrs = 2;
+        e = cudaLaunchKernelEx(&cfg, kern, P, g);
+        if (with_pdl && (e == cudaErrorNotSupported || e == cudaErrorInvalidValue)) {
+            (void)cudaGetLastError();
+            attr[0] = attr[1]; cfg.numAttrs = 1;
+            e = cudaLaunchKernelEx(&cfg, kern, P, g);
+            if (e == cudaSuccess) c_pdl.store(0);     // the pair is what this system refuses
+        }
+        if (e == cudaSuccess) { v_dev = dev; v_smem = smem; }
     }
     if (e == cudaErrorCooperativeLaunchTooLarge) {   // fewer SMs at hand than the device reports: the one-CTA-per-row kernel serves
         (void)cudaGetLastError();
