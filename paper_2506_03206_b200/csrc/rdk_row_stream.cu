@@ -504,10 +504,10 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
     };
     // The load warp sets up the ring by itself and starts the first rows' copies right away, so that HBM's first
     // answer travels while the rest of the CTA is still setting up: it initialises the ring's barriers, gives the
-    // parts of the stages that no copy writes their neutral values (beyond the vocabulary and the 16 spare bytes of
-    // every stage: weight 0; the drafter regions start out as weight 0 too -- slots beyond a copy keep whatever an
-    // earlier row left there, and are masked), and issues the first NS rows.
-    const int pre_rows = min(g.NS, rows_g);
+    // parts of the target slices that no copy writes the weight 0 (beyond the vocabulary, and the 16 spare bytes of
+    // every stage that padded gathers point at), and issues the first row.  The drafter regions need no such
+    // care: every slot a copy did not fill (or filled with a neighbouring segment's values) is masked where it is read.
+    const int pre_rows = min(1, rows_g);     // a single warp takes about 0.6 us to issue a row: the others follow the barrier
     if (warp == kWLoad) {
         if (lane == 0) {
             for (int k = 0; k < g.NS; ++k) {
@@ -517,15 +517,13 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         {
-            const uint32_t fill16 = KIND == RDK_LOGITS ? (sizeof(TY) == 2 ? 0xff80ff80u : 0xff800000u) : 0u;      // -inf, or 0
-            const uint32_t ninf16 = sizeof(TZ) == 2 ? 0xff80ff80u : 0xff800000u;
+            const uint32_t ninf16 = sizeof(TZ) == 2 ? 0xff80ff80u : 0xff800000u;      // -inf
             const uint32_t z0 = zbytes, z1 = zslice + 16u;        // [end of the copied vectors, spare bytes included)
             for (int k = 0; k < g.NS; ++k) {
                 const uint32_t base = dsm_a + (uint32_t)k * stage;
+#pragma unroll 8
                 for (uint32_t o = z0 + 16u * lane; o < z1; o += 512u)
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + o), "r"(ninf16) : "memory");
-                for (uint32_t o = z1 + 16u * lane; o < stage; o += 512u)
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + o), "r"(fill16) : "memory");
             }
         }
         __syncwarp();
@@ -867,7 +865,7 @@ rdk_stream_kernel(const RowParams P, const StreamGeo g) {
         }
     } else {
         // ================================ load warp =====================================================
-        // the first rows went out during the set-up; one row per stage as the streaming warps release them
+        // the first row went out during the set-up; one row per stage as the streaming warps release them
         for (int it = pre_rows; it < rows_g; ++it) load_row();
         if (ld_volatile_s32(&fail)) {
             // A wait gave up somewhere, so nobody may have waited for the last copies: let them land before
