@@ -364,6 +364,16 @@ def bench_workload(ctx: Ctx, name: str, steps: int, warmup: int, prior: bool, he
     kern_ms = ctx.timed_repeats(kernel_fn, steps, warm_ms)
     sampler.stop()
     B.check_status_word(outs[0], f"bench step {name}")
+    burst_ms = None
+    if exact:
+        # The same call under the condition the burst peak was measured in: short runs (about 20 ms) that start
+        # from an idle device, before the power cap pulls the clocks down; the loops above are the sustained case.
+        bursts = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            time.sleep(1.0)
+            bursts.append(ctx.timed(kernel_fn, 50) / 50)
+        burst_ms = sorted(bursts)[1]
     ms, spread = median_and_spread(loop_ms)
     kms, kspread = median_and_spread(kern_ms)
     kernel_ms = kms / steps
@@ -416,7 +426,10 @@ def bench_workload(ctx: Ctx, name: str, steps: int, warmup: int, prior: bool, he
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["tensor"], "unit": "TFLOP/s",
                     "frac": achieved / peaks["tensor"], "traffic": None, "kernel_ms": kernel_ms, "flops_per_launch": flops,
                     "peak_source": peaks["source"], "frac_of_sustained_peak": achieved / peaks["tensor_sustained"],
-                    "tensor_pipe_pct_of_measured_peak": 100.0 * achieved / peaks["tensor"], "kernels": kernels}
+                    "tensor_pipe_pct_of_measured_peak": 100.0 * achieved / peaks["tensor"], "kernels": kernels,
+                    "burst": {"kernel_ms": burst_ms, "achieved": flops / (burst_ms * 1e-3) / 1e12,
+                              "frac_of_burst_peak": flops / (burst_ms * 1e-3) / 1e12 / peaks["tensor"],
+                              "how": "median of 3 runs of 50 calls, each run after 1 s of idle"}}
     else:
         algo_bytes = rows * row_bytes
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9

@@ -924,23 +924,33 @@ rdk_draw_kernel(const RowParams P, const int nseg, const int Lw) {
 
     if (warp < 3) {   // fp64 prefix sums over the segments: warp 0 those of w, warp 1 of max(0, p - q~), warp 2 of p
         double* cdf = warp == 0 ? cdfW : (warp == 1 ? cdfR : cdfP);
-        double carry = 0.0;
-        for (int base = 0; base < nseg; base += 32) {
-            const int s = base + lane;
-            double x = 0.0;
-            if (s < nseg) {
-                const float4 v = __ldcg(reinterpret_cast<const float4*>(rec + 16) + s);
-                x = (double)(warp == 0 ? v.x : (warp == 1 ? v.z : v.w));
-            }
+        // a lane takes K consecutive segments (all loads first), sums them up in order, and one scan over
+        // the lanes' totals places its run
+        constexpr int K = kMaxSeg / 32;
+        const int per = (nseg + 31) >> 5, s0 = lane * per;
+        float v[K];
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double a = __shfl_up_sync(0xffffffffu, x, o);
-                if (lane >= o) x += a;
+        for (int k = 0; k < K; ++k) {
+            v[k] = 0.f;
+            if (k < per && s0 + k < nseg) {
+                const float4 r4 = __ldcg(reinterpret_cast<const float4*>(rec + 16) + s0 + k);
+                v[k] = warp == 0 ? r4.x : (warp == 1 ? r4.z : r4.w);
             }
-            x += carry;
-            carry = __shfl_sync(0xffffffffu, x, 31);
-            if (s < nseg) cdf[s] = x;
         }
+        double run[K], x = 0.0;
+#pragma unroll
+        for (int k = 0; k < K; ++k) { x += (double)v[k]; run[k] = x; }
+        double incl = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double a = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += a;
+        }
+        double before = __shfl_up_sync(0xffffffffu, incl, 1);      // the previous lane's last value, so the sequence never steps back
+        if (lane == 0) before = 0.0;
+#pragma unroll
+        for (int k = 0; k < K; ++k)
+            if (k < per && s0 + k < nseg) cdf[s0 + k] = before + run[k];
     } else if (warp == 3) {   // alpha = sum over the segments of sum min(p, q~)
         float alpha_l = 0.f;
         for (int s = lane; s < nseg; s += 32) alpha_l += __ldcg(reinterpret_cast<const float4*>(rec + 16) + s).y;
