@@ -556,6 +556,36 @@ def acceptance_report(ctx: Ctx, name: str = "T1"):
                     "formula moves about theta / N of the drafter's mass off the kept ids, so (b) and (c) differ by about that"}
 
 
+def acceptance_exact_vs_linear(ctx: Ctx, name: str = "C5", rows: int = 256):
+    """Mean acceptance rate of exact RDK (w = M^T q', Algorithm 1 step 2, bf16 affinity on the tensor cores), of the
+    first-order formula (Eq. rdk-taylor) and of TLI on the same rows of the exact workload, all from the library's
+    kernels; `rows` rows of the workload (the affinity matrix is the workload's own)."""
+    torch, B, W = ctx.torch, ctx.B, ctx.W
+    cfg = W.CONFIGS[name]
+    inp = W.make_inputs(cfg, device=str(ctx.dev), with_embeddings=True)
+    kind = B.RDK_PROBS if cfg.drafter_kind == "probs" else B.RDK_LOGITS
+    batch = max(1, min(cfg.batch, rows // cfg.positions))
+    n_rows = batch * cfg.positions
+    tgt, dr, un = inp["target"][:n_rows], inp["drafter"][:n_rows], inp["uniforms"][:n_rows]
+    kid = inp["kept_ids"].long()
+    index = B.rdk_prepare_ids(inp["kept_ids"], cfg.N)
+    M = B.rdk_build_affinity(inp["embeddings"], inp["kept_ids"], cfg.tau, B.RDK_AFF_BF16_COLS)
+    w, _, _ = B.rdk_redistribute_exact(index, dr, M, batch, cfg.positions, kind)
+    exact = B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, tgt, None, w, un, batch, cfg.positions, kind)
+    linear = B.rdk_sample_and_verify(index, B.RDK_MODE_LINEAR, tgt, dr, None, un, batch, cfg.positions, kind)
+    q = dr.float() if kind == B.RDK_PROBS else torch.softmax(dr.float(), dim=-1)
+    wt = torch.zeros(n_rows, cfg.N, dtype=torch.float32, device=ctx.dev)
+    wt[:, kid] = q
+    tli = B.rdk_sample_and_verify(index, B.RDK_MODE_PRECOMPUTED_W, tgt, None, wt, un, batch, cfg.positions, kind)
+    torch.cuda.synchronize()
+    for o in (exact, linear, tli):
+        B.check_status_word(o, f"acceptance report {name}")
+    mean = lambda t: float(t.double().mean())
+    return {"workload": f"{name}: N={cfg.N}, n={cfg.n}, {n_rows} rows, affinity = soft-max of cosine similarities at tau={cfg.tau}",
+            "mean_alpha": {"tli": mean(tli["alpha"]), "taylor_rdk": mean(linear["alpha"]), "exact_rdk": mean(exact["alpha"])},
+            "mean_l1_exact_vs_tli": float((w / w.sum(-1, keepdim=True) - wt / wt.sum(-1, keepdim=True)).abs().sum(-1).double().mean())}
+
+
 def run_ours(args):
     import torch
 
@@ -600,6 +630,8 @@ def run_ours(args):
     acceptance = None
     if rank == 0 and not args.prior and (not args.only or args.workload == "T1"):
         acceptance = acceptance_report(ctx)
+        if not args.only:
+            acceptance["exact_vs_linear"] = acceptance_exact_vs_linear(ctx)
 
     if rank != 0:
         if dist is not None:
