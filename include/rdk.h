@@ -158,7 +158,12 @@ int rdk_prepare_ids(const int32_t* kept_ids, int32_t n, int32_t N, void* kept_in
  *   M_out        device, layout / ld as in rdk_affinity (data member is ignored; M_out is used)
  *   ws           device workspace of rdk_build_affinity_workspace_bytes(N, n, d) bytes
  * Arithmetic: fp32 dot products and soft-max; the result is rounded to bf16 (nearest even) only
- * when it is stored in the bf16 layout.
+ * when it is stored in the bf16 layout.  bf16 embeddings (d >= 64, 16-byte aligned rows) going to the
+ * bf16 layout take the tensor cores for the dot products (bf16 products are exact, accumulation in
+ * fp32), in chunks of 2048 kept rows through an fp32 scratch [N, 2048] inside the workspace; every
+ * other combination uses fp32 FMAs.  Both routes compute the same quantity.  If a bounded wait
+ * inside the tensor-core kernel expires (the call has no status word), element [0, 0] of M_out is
+ * set to NaN.
  * ------------------------------------------------------------------------------------------- */
 size_t rdk_build_affinity_workspace_bytes(int32_t N, int32_t n, int32_t d);
 int rdk_build_affinity(const void* embeddings, int32_t emb_dtype, int32_t d, int64_t emb_row_stride,

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librdk_b200.so")
-SOURCES = ["rdk_api.cu", "rdk_ids.cu", "rdk_row.cu", "rdk_row_stream.cu", "rdk_emit.cu", "rdk_affinity.cu", "rdk_exact.cu", "rdk_exact_tc.cu"]
+SOURCES = ["rdk_api.cu", "rdk_ids.cu", "rdk_row.cu", "rdk_row_stream.cu", "rdk_emit.cu", "rdk_affinity.cu", "rdk_affinity_tc.cu", "rdk_exact.cu", "rdk_exact_tc.cu"]
 
 
 def _nvcc() -> str:

@@ -112,13 +112,20 @@ aff_rows_kernel(const float* __restrict__ Et, const int32_t* __restrict__ ids, i
     }
 }
 
+// the tensor-core route (bf16 embeddings into the bf16 layout)
+size_t affinity_tc_workspace_bytes(int N, int n, int d);
+bool affinity_tc_eligible(const void* embeddings, int emb_dtype, int d, long long estride, int layout);
+int build_affinity_tc(const __nv_bfloat16* E, int d, long long estride, const int32_t* ids, int n, int N, float tau,
+                      __nv_bfloat16* Mt, long long ld, void* ws, cudaStream_t s);
+
 }  // namespace rdk
 
 using namespace rdk;
 
 extern "C" size_t rdk_build_affinity_workspace_bytes(int32_t N, int32_t n, int32_t d) {
     if (N < 1 || n < 1 || d < 1) return 0;
-    return idx_align((size_t)N * d * sizeof(float));
+    const size_t fma = idx_align((size_t)N * d * sizeof(float)), tc = affinity_tc_workspace_bytes(N, n, d);
+    return fma > tc ? fma : tc;          // either route may serve the call
 }
 
 extern "C" int rdk_build_affinity(const void* embeddings, int32_t emb_dtype, int32_t d, int64_t emb_row_stride,
@@ -153,6 +160,9 @@ extern "C" int rdk_build_affinity(const void* embeddings, int32_t emb_dtype, int
     const int st = check_arch();
     if (st != RDK_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (affinity_tc_eligible(embeddings, emb_dtype, d, estride, M_desc->layout))
+        return build_affinity_tc(static_cast<const __nv_bfloat16*>(embeddings), d, estride, kept_ids, n, N, tau,
+                                 static_cast<__nv_bfloat16*>(M_out), M_desc->ld, ws, s);
     float* Et = static_cast<float*>(ws);
     const int wpb = 8;
     if (emb_dtype == RDK_F32)

@@ -72,6 +72,33 @@ def test_build_affinity_bf16_cols_and_dropped_rows():
     assert np.all(got[3] == 0) and np.all(got[17] == 0)
 
 
+@pytest.mark.parametrize("N,n,d", [(3000, 300, 72), (4100, 2300, 128), (700, 64, 64)])
+def test_build_affinity_on_the_tensor_cores(N, n, d):
+    """bf16 embeddings of dimension >= 64 into the bf16 layout: the dot products run on the tensor cores (ragged
+    embedding dimension, ragged tiles, more kept rows than one chunk, ids outside the vocabulary), compared with the
+    checker's matrix rounded to bf16: equal except where fp32 arithmetic lands on the other side of a rounding
+    boundary (then the neighbouring bf16 number)."""
+    rdk = _rdk()
+    B = rdk.binding
+    cfg = W.tiny_config(N=N, n=n, emb_dim=d, dtype="bf16", seed=N + d)
+    inp = W.make_inputs(cfg, with_embeddings=True)
+    assert inp["embeddings"].dtype == torch.bfloat16
+    ids = inp["kept_ids"].clone()
+    ids[5] = -3
+    ids[n - 2] = N
+    M_ref = O.build_affinity(W.to_f64(inp["embeddings"]), ids.numpy(), cfg.tau)
+    M = rdk.rdk_build_affinity(inp["embeddings"].cuda(), ids.cuda(), cfg.tau, B.RDK_AFF_BF16_COLS)
+    torch.cuda.synchronize()
+    got = M["data"][:, :n].cpu().double().numpy().T
+    assert not np.isnan(got).any()
+    M_rnd = O.round_to_bf16(M_ref)
+    assert np.mean(got == M_rnd) >= 0.99
+    assert np.all(np.abs(got - M_rnd) <= 2.0 ** -7 * M_rnd + 1e-38)
+    assert np.all(np.abs(got - M_ref) <= (2.0 ** -8 + 1e-4) * M_ref + 1e-38)
+    assert np.all(got[5] == 0) and np.all(got[n - 2] == 0)
+    assert np.all(np.abs(got.sum(axis=1)[[0, 1, n - 1]] - 1.0) < 5e-3)
+
+
 def _flip_allowance(qp, Mcols):
     """The left operand q' is rounded to bf16 on the GPU from an fp32 value and in the checker from a
     float64 value.  An element whose exact value lies within fp32 rounding error (2e-6 relative) of a
