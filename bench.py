@@ -177,12 +177,12 @@ def _cpu_baseline_exact(cfg, name: str, rows: int = 256, cols: int = 4096):
     t_contract = (time.perf_counter() - t0) * (cfg.N / cols)
     t0 = time.perf_counter()
     for r in range(rows):
-        O.rdk_row(z[r], None, kappa, u[r], "given", w_given=np.tile(wc[r], cfg.N // cols))
+        O.rdk_row(z[r], None, kappa, u[r], "given", w_given=np.resize(wc[r], cfg.N))
     t_sample = time.perf_counter() - t0
     dt = t_contract + t_sample
     return {"value": rows / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": (f"{rows} rows of {name}: oracle.redistribute_exact on {cols} of {cfg.N} seeded columns of the checker's "
-                       f"bf16-rounded affinity matrix, time scaled by {cfg.N // cols} ({t_contract:.1f} s), plus oracle.rdk_row "
+                       f"bf16-rounded affinity matrix, time scaled by {cfg.N / cols:.1f} ({t_contract:.1f} s), plus oracle.rdk_row "
                        f"(mode 'given') on full-length weights ({t_sample:.1f} s); float64 numpy, one thread")}
 
 
@@ -632,6 +632,8 @@ def run_ours(args):
         acceptance = acceptance_report(ctx)
         if not args.only:
             acceptance["exact_vs_linear"] = acceptance_exact_vs_linear(ctx)
+    if rank == 0 and args.workload == "X2":
+        acceptance = {"exact_vs_linear": acceptance_exact_vs_linear(ctx, "X2", rows=W.CONFIGS["X2"].rows)}
 
     if rank != 0:
         if dist is not None:
@@ -659,7 +661,7 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["C2", "C3", "C4", "C5", "T1"], default=WORKLOAD,
+    ap.add_argument("--workload", choices=["C2", "C3", "C4", "C5", "T1", "X2"], default=WORKLOAD,
                     help="the headline workload of the line (default C2, the one the metric is quoted on); the others "
                          "ride along under \"workloads\"")
     ap.add_argument("--only", action="store_true", help="time the headline workload only (profiling runs)")

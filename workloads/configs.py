@@ -76,6 +76,12 @@ CONFIGS: Dict[str, RDKConfig] = {
     "C5": RDKConfig("C5", N=32768, n=8192, batch=1024, positions=1, dtype="bf16", path="exact",
                     kept_rule="uniform", sigma=2.0, zipf_bias=False, rho=0.8, emb_dim=128, trials=1,
                     drafter_kind="probs", seed=105),
+    # The exact redistribution at the Llama-3-scale shape of C2 (Sec. 4 sets it aside as O(N^2)): the
+    # same vocabulary, kept ids, logits and embeddings as C2, through M^T q' instead of Eq. rdk-taylor.
+    # Not one of the benchmark configurations; bench.py --workload X2 times it.
+    "X2": RDKConfig("X2", N=128256, n=32064, batch=64, positions=5, dtype="bf16", path="exact",
+                    kept_rule="zipf", sigma=3.0, zipf_bias=True, rho=0.0, emb_dim=256, trials=1,
+                    seed=102),
 }
 
 
