@@ -87,7 +87,13 @@ def test_build_affinity_on_the_tensor_cores(N, n, d):
     ids[5] = -3
     ids[n - 2] = N
     M_ref = O.build_affinity(W.to_f64(inp["embeddings"]), ids.numpy(), cfg.tau)
-    M = rdk.rdk_build_affinity(inp["embeddings"].cuda(), ids.cuda(), cfg.tau, B.RDK_AFF_BF16_COLS)
+    emb = inp["embeddings"].cuda()
+    if d == 72:      # rows inside a wider buffer: a row stride of 80 elements (16-byte aligned rows)
+        wide = torch.zeros(N, 80, dtype=torch.bfloat16, device="cuda")
+        wide[:, :d] = emb
+        emb = wide[:, :d]
+        assert emb.stride(0) == 80
+    M = rdk.rdk_build_affinity(emb, ids.cuda(), cfg.tau, B.RDK_AFF_BF16_COLS)
     torch.cuda.synchronize()
     got = M["data"][:, :n].cpu().double().numpy().T
     assert not np.isnan(got).any()
