@@ -37,8 +37,8 @@ MIN_TIMED_SECONDS = 0.5      # the K-step loop is repeated until at least this m
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources with this hash.
-NCU_TRAFFIC = {"sources_sha256": "1dd8cc61b388521b27af0288dc93da6eaafe5f60715cb810fd25ef8a4a6df0ac",
-               "bytes_per_launch": {"C2": 107126528, "C3": 586670080}}
+NCU_TRAFFIC = {"sources_sha256": "1e0aa2b1d5ccce991f824bee5f0645738ce82e870d36d720dafa90eb37320f60",
+               "bytes_per_launch": {"C2": 106771456, "C3": 586242560}}
 KERNEL_SOURCES = ("rdk_row_stream.cu", "rdk_row.cuh", "rdk_common.cuh")
 
 

@@ -201,33 +201,15 @@ template <> struct MaxAcc<__nv_bfloat16> {
     }
 };
 
-// 2^t for a pair, t <= 0, on the FMA pipe instead of the special-function unit: t = n + f with n the
-// nearest integer (the low bits of t + 1.5 * 2^23) and |f| <= 1/2, 2^f by a degree-5 polynomial (relative
-// error 2.4e-7, that of ex2.approx), 2^n by adding n to the exponent field.  Below -126 the result is
-// about 1e-38 in place of 0.
-__device__ __forceinline__ float2 ex2_poly2(float2 t) {
-    t.x = fmaxf(t.x, -126.f); t.y = fmaxf(t.y, -126.f);
-    const float2 r = fadd2(t, splat(12582912.f));
-    const float2 n = fadd2(r, splat(-12582912.f));
-    const float2 f = ffma2(n, splat(-1.f), t);
-    float2 p = ffma2(splat(0.001327647129073739f), f, splat(0.009675540961325169f));
-    p = ffma2(p, f, splat(0.05550713092088699f));
-    p = ffma2(p, f, splat(0.24022120237350464f));
-    p = ffma2(p, f, splat(0.6931469440460205f));
-    p = ffma2(p, f, splat(1.0000001192092896f));
-    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23)),
-                       __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23)));
-}
-
-// sum of e = 2^(z log2e + off) over the logits of one 16-byte vector, two packed accumulators.  For bf16
-// logits one pair in four takes the polynomial: the sweep is bound by the special-function unit (16
-// results per clock per SM), and a quarter is what the issue slots have room for.
+// sum of e = 2^(z log2e + off) over the logits of one 16-byte vector, two packed accumulators.  (Evaluating a
+// share of the exponentials by a polynomial on the FMA pipe relieves the special-function unit but costs issue
+// slots, which are the scarcer resource in this kernel: measured, it does not pay.)
 template <typename TZ> __device__ __forceinline__ void exp_sum_vec(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb);
 template <> __device__ __forceinline__ void exp_sum_vec<__nv_bfloat16>(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb) {
     const float2 e0 = ex2_2(ffma2(make_float2(bf16_lo(q.x), bf16_hi(q.x)), scale, off));
     const float2 e1 = ex2_2(ffma2(make_float2(bf16_lo(q.y), bf16_hi(q.y)), scale, off));
     const float2 e2 = ex2_2(ffma2(make_float2(bf16_lo(q.z), bf16_hi(q.z)), scale, off));
-    const float2 e3 = ex2_poly2(ffma2(make_float2(bf16_lo(q.w), bf16_hi(q.w)), scale, off));
+    const float2 e3 = ex2_2(ffma2(make_float2(bf16_lo(q.w), bf16_hi(q.w)), scale, off));
     Ea = fadd2(Ea, e0); Eb = fadd2(Eb, e1); Ea = fadd2(Ea, e2); Eb = fadd2(Eb, e3);
 }
 template <> __device__ __forceinline__ void exp_sum_vec<float>(uint4 q, float2 scale, float2 off, float2& Ea, float2& Eb) {
